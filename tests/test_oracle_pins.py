@@ -1,0 +1,618 @@
+"""Pins for the CPU oracle: closed forms, brute force, invariants and a second,
+independent formulation.  Each test is chosen so that a plausible mistake in the
+oracle (dropped term, wrong sign or index, transposed operand) fails it.
+No GPU is involved."""
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.linalg
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")
+
+
+def golden():
+    out = {}
+    with open(GOLDEN) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, v = line.split()
+            out[k] = float(v)
+    return out
+
+
+# ----------------------------------------------------------------------------
+# Eq. 2 / Eq. 3: static horizon
+# ----------------------------------------------------------------------------
+
+def test_horizon_closed_form_values():
+    gc = golden()
+    a, eps = gc["gate_logit_a"], gc["epsilon"]
+    # softplus(-0.3) and ln(1e-3) from tables of the elementary functions
+    g, Hs = oracle.horizon([0.0], [0.0], a=a, eps=eps)
+    assert g[0] == pytest.approx(-0.5543552444685271, rel=1e-14)
+    assert Hs[0] == pytest.approx(12.46088198480878, rel=1e-13)
+    # rate 0.1 -> ten times the horizon
+    _, Hs01 = oracle.horizon([np.float32(math.log(0.1))], [0.0], a=a, eps=eps)
+    rate = math.exp(float(np.float32(math.log(0.1))))
+    assert Hs01[0] == pytest.approx(12.46088198480878 / rate, rel=1e-13)
+    # Section 3.3: a = -0.3 gives a longer horizon than a = 0 (ln 2 = softplus(0))
+    _, Hs0 = oracle.horizon([0.0], [0.0], a=0.0, eps=eps)
+    assert Hs0[0] == pytest.approx(6.907755278982137 / 0.6931471805599453, rel=1e-13)
+    assert Hs[0] > Hs0[0]
+
+
+def test_horizon_defining_property():
+    # A unit with constant log-decay g and beta = 0 has decayed to exactly eps after H_s tokens.
+    rng = np.random.default_rng(0)
+    A_log = rng.normal(size=64).astype(np.float32)
+    dt = rng.normal(size=64).astype(np.float32)
+    g, Hs = oracle.horizon(A_log, dt, a=-0.3, eps=1e-3)
+    assert np.all(g < 0) and np.all(Hs > 0)
+    np.testing.assert_allclose(np.exp(g * Hs), 1e-3, rtol=1e-12)
+    # dt_bias enters through softplus: large positive bias -> g ~ -(a + bias) * exp(A_log)
+    g2, _ = oracle.horizon([0.0], [40.0], a=-0.3)
+    assert g2[0] == pytest.approx(-39.7, rel=1e-12)
+    # A_log enters through exp, multiplicatively
+    g3, _ = oracle.horizon([1.0], [0.0], a=-0.3)
+    assert g3[0] == pytest.approx(-math.e * 0.5543552444685271, rel=1e-13)
+
+
+# ----------------------------------------------------------------------------
+# Eq. 7: replay windows
+# ----------------------------------------------------------------------------
+
+def test_replay_window_examples():
+    assert oracle.replay_window_unit(12.46, 64) == 16
+    assert oracle.replay_window_unit(3.0, 64) == 4        # low clamp
+    assert oracle.replay_window_unit(0.3, 64) == 4
+    assert oracle.replay_window_unit(16.0, 64) == 16      # exact power maps to itself
+    assert oracle.replay_window_unit(16.000001, 64) == 32
+    assert oracle.replay_window_unit(1000.0, 128) == 128  # high clamp
+    assert oracle.replay_window_unit(64.0, 64) == 64
+
+
+def test_replay_window_matches_table8_reading():
+    # Table 8: replayed tokens per hit equal W_max (16.0, 64.0) or fall just below it
+    # (prefix clipping).  With a threshold plan every omitted unit has H_s <= W_max, so the
+    # high clamp never bites, and as soon as one omitted unit has H_s > W_max/2 the window is W_max.
+    gc = golden()
+    rng = np.random.default_rng(1)
+    for w_max in (16, 64, 128, 512, 1024):
+        assert gc[f"replay_tokens_wmax_{w_max}"] <= w_max
+        rates = np.exp(rng.uniform(math.log(1e-3), 0.0, size=(2, 4 * 32))).astype(np.float32)
+        p = oracle.plan(oracle.KDA, 2, 4, 32, np.log(rates), np.zeros_like(rates), w_max=float(w_max))
+        omitted = p.mask == 0
+        assert np.all(p.Hs[omitted] <= w_max)
+        assert np.all(p.W_u[omitted] <= w_max)
+        if np.any(p.Hs[omitted] > w_max / 2):
+            assert p.W_replay == w_max
+        # brute force of Eq. 7
+        want = 0.0
+        for h in p.Hs[omitted]:
+            w = 2.0 ** math.ceil(math.log2(h))
+            want = max(want, min(max(w, 4.0), float(w_max)))
+        assert p.W_replay == want
+    # no omitted units -> no replay
+    p = oracle.plan(oracle.GDN, 1, 4, 1, np.full(4, -20.0, np.float32), np.zeros(4, np.float32), w_max=16.0)
+    assert p.mask.all() and p.W_replay == 0
+
+
+# ----------------------------------------------------------------------------
+# Section 4.1 selection, Appendix B offsets, Eq. 6 ratios
+# ----------------------------------------------------------------------------
+
+def _brute_threshold(Hs, w_max):
+    return (Hs > w_max).astype(np.uint8)
+
+
+def test_threshold_rule_is_strict_and_offsets_are_prefix_sums():
+    # put one unit exactly on the threshold: H_s == W_max must be omitted
+    base = 12.46088198480878
+    A_log = np.zeros((3, 8), np.float32)
+    A_log[0, :4] = np.log(np.float32(0.01))
+    A_log[1, :] = np.log(np.float32(2.0))
+    A_log[2, 1::2] = np.log(np.float32(0.001))
+    _, Hs = oracle.horizon(A_log, np.zeros_like(A_log))
+    w_max = float(Hs.reshape(3, 8)[0, 7])            # equals `base`
+    assert w_max == pytest.approx(base)
+    p = oracle.plan(oracle.GDN, 3, 8, 1, A_log, np.zeros_like(A_log), w_max=w_max)
+    np.testing.assert_array_equal(p.mask, _brute_threshold(Hs.reshape(3, 8), w_max))
+    assert p.mask[0, 7] == 0 and p.mask[0, 0] == 1
+    np.testing.assert_array_equal(p.r_l, [4, 0, 4])
+    np.testing.assert_array_equal(p.o_l, [0, 4, 4, 8])
+    assert p.sum_r == p.o_l[-1] == 8 and p.sum_n == 24 and p.R_max == 4
+    # Eq. 6 and Appendix B closed forms
+    assert p.C_temp_rag == pytest.approx(24 / 8)
+    assert p.C_temp_pad == pytest.approx(24 / (3 * 4))
+    assert p.C_temp_rag / p.C_temp_pad == pytest.approx(p.R_max / p.r_l.mean())
+
+
+def test_threshold_monotone_in_wmax():
+    rng = np.random.default_rng(2)
+    rates = np.exp(rng.uniform(math.log(1e-3), 0.0, size=(4, 64))).astype(np.float32)
+    prev = None
+    for w_max in (4, 16, 64, 128, 512, 1024, 1e9):
+        p = oracle.plan(oracle.KDA, 4, 2, 32, np.log(rates), np.zeros_like(rates), w_max=float(w_max))
+        if prev is not None:
+            assert np.all(p.mask <= prev)       # raising W_max never un-omits a unit
+        prev = p.mask
+    assert prev.sum() == 0
+
+
+def test_top_ratio_brute_force_and_ties():
+    rng = np.random.default_rng(3)
+    L, H, D = 3, 4, 16
+    rates = np.exp(rng.uniform(math.log(1e-3), 0.0, size=(L, H * D))).astype(np.float32)
+    rates[0, 5] = rates[0, 9] = rates[0, 20]      # exact ties inside one group
+    A_log = np.log(rates)
+    _, Hs = oracle.horizon(A_log, np.zeros_like(A_log))
+    Hs = Hs.reshape(L, H * D)
+    for scope, group in ((oracle.SCOPE_HEAD, D), (oracle.SCOPE_LAYER, H * D), (oracle.SCOPE_MODEL, L * H * D)):
+        for ratio in (0.0, 0.2, 0.38, 0.4, 0.5, 1.0):
+            p = oracle.plan(oracle.KDA, L, H, D, A_log, np.zeros_like(A_log), sel=oracle.SEL_TOP_RATIO,
+                            keep_ratio=ratio, scope=scope)
+            want = np.zeros(L * H * D, np.uint8)
+            flat = Hs.ravel()
+            r = min(group, max(0, math.ceil(ratio * group - 1e-9)))
+            for base in range(0, flat.size, group):
+                # stable sort on -H_s: largest first, lower index first among equals
+                order = np.argsort(-flat[base:base + group], kind="stable")
+                want[base + order[:r]] = 1
+            np.testing.assert_array_equal(p.mask.ravel(), want)
+            assert p.sum_r == want.sum()
+            np.testing.assert_array_equal(np.diff(p.o_l), p.r_l)
+    # the benchmark's tiny configuration: 40 % of 64 channels per head -> 26
+    p = oracle.plan(oracle.KDA, 1, 4, 64, np.log(rng.uniform(0.01, 1, (1, 256)).astype(np.float32)),
+                    np.zeros((1, 256), np.float32), sel=oracle.SEL_TOP_RATIO, keep_ratio=0.4,
+                    scope=oracle.SCOPE_HEAD)
+    np.testing.assert_array_equal(p.mask.reshape(4, 64).sum(1), [26] * 4)
+
+
+def test_random_selector_is_count_matched_and_seeded():
+    rng = np.random.default_rng(4)
+    rates = np.exp(rng.uniform(math.log(1e-3), 0.0, size=(5, 96))).astype(np.float32)
+    A_log = np.log(rates)
+    base = oracle.plan(oracle.KDA, 5, 3, 32, A_log, np.zeros_like(A_log), w_max=64.0)
+    masks = []
+    for seed in (1234, 2027, 3407):
+        p = oracle.plan(oracle.KDA, 5, 3, 32, A_log, np.zeros_like(A_log), w_max=64.0, randomize=True, seed=seed)
+        np.testing.assert_array_equal(p.r_l, base.r_l)     # same r_l per layer
+        masks.append(p.mask.copy())
+        p2 = oracle.plan(oracle.KDA, 5, 3, 32, A_log, np.zeros_like(A_log), w_max=64.0, randomize=True, seed=seed)
+        np.testing.assert_array_equal(p.mask, p2.mask)
+    assert not np.array_equal(masks[0], masks[1])
+    assert not np.array_equal(masks[0], base.mask)
+    # uniformity smoke: over many seeds every unit of a layer is picked about r/n of the time
+    hits = np.zeros(96)
+    n_seeds = 400
+    for seed in range(n_seeds):
+        p = oracle.plan(oracle.KDA, 5, 3, 32, A_log, np.zeros_like(A_log), w_max=64.0, randomize=True, seed=seed)
+        hits += p.mask[2]
+    frac = base.r_l[2] / 96
+    assert abs(hits.mean() / n_seeds - frac) < 1e-12
+    assert np.all(np.abs(hits / n_seeds - frac) < 0.12)
+
+
+def test_slot_budget_and_checkpoint_accounting_match_paper():
+    gc = golden()
+    tp = int(gc["tp_degree"])
+    # Kimi-KDA: 20 layers x 32 heads x 128x128 fp32 temporal state, sharded over TP8,
+    # plus three bf16 convolution taps over q, k, v channels per rank.
+    kda_temporal = int(gc["kimi_kda_layers"]) * 32 * 128 * 128 * 4 // tp
+    kda_conv = int(gc["kimi_kda_layers"]) * 3 * (3 * 32 * 128) // tp * 2
+    assert (kda_temporal + kda_conv) * int(gc["dense_physical_slots"]) == int(gc["budget_bytes_kimi_kda"])
+    assert oracle.slot_budget(int(gc["budget_bytes_kimi_kda"]), [kda_temporal] * tp, kda_conv) == gc["dense_deployable_slots"]
+    # Qwen-GDN: 36 layers x 32 value-head states, 16 key heads
+    gdn_temporal = int(gc["qwen_gdn_layers"]) * 32 * 128 * 128 * 4 // tp
+    gdn_conv = int(gc["qwen_gdn_layers"]) * 3 * (2 * 16 * 128 + 32 * 128) // tp * 2
+    assert (gdn_temporal + gdn_conv) * int(gc["dense_physical_slots"]) == int(gc["budget_bytes_qwen_gdn"])
+    assert oracle.slot_budget(int(gc["budget_bytes_qwen_gdn"]), [gdn_temporal] * tp, gdn_conv) == gc["dense_deployable_slots"]
+    # the most loaded rank limits the count
+    assert oracle.slot_budget(1000, [90, 240, 10], 10) == 1000 // 250 - 1
+    # Eq. 6 complete-checkpoint ratio: everything retained -> 1; half retained, no conv -> 2
+    A_log = np.array([[-9.0, -9.0, 3.0, 3.0]], np.float32)
+    p = oracle.plan(oracle.GDN, 1, 4, 1, A_log, np.zeros_like(A_log), w_max=16.0, unit_bytes=65536, conv_bytes=0)
+    assert p.sum_r == 2 and p.C_temp_rag == 2.0 and p.C_ckpt_rag == 2.0
+    p = oracle.plan(oracle.GDN, 1, 4, 1, A_log, np.zeros_like(A_log), w_max=16.0, unit_bytes=65536, conv_bytes=131072)
+    assert p.C_ckpt_rag == pytest.approx((4 * 65536 + 131072) / (2 * 65536 + 131072))
+    p = oracle.plan(oracle.GDN, 1, 4, 1, A_log, np.zeros_like(A_log), w_max=0.0, unit_bytes=65536, conv_bytes=777)
+    assert p.sum_r == 4 and p.C_ckpt_rag == 1.0 and p.C_temp_pad == 1.0
+
+
+# ----------------------------------------------------------------------------
+# pack / restore invariants
+# ----------------------------------------------------------------------------
+
+def _state_with_specials(rng, shape):
+    s = rng.normal(size=shape).astype(np.float32)
+    bits = s.view(np.uint32).ravel()
+    specials = np.array([0x80000000, 0x00000001, 0x807FFFFF, 0x7F800000, 0xFF800000, 0x7FC00001, 0xFFC12345],
+                        np.uint32)
+    idx = rng.choice(bits.size, size=min(bits.size, 40), replace=False)
+    bits[idx] = specials[np.arange(idx.size) % specials.size]
+    return s
+
+
+@pytest.mark.parametrize("unit_words,n_l", [(8, 24), (32, 5)])
+def test_pack_is_concatenation_and_restore_is_masking(unit_words, n_l):
+    rng = np.random.default_rng(5)
+    L, n_req, n_slots = 3, 4, 6
+    mask = (rng.random((L, n_l)) < 0.4).astype(np.uint8)
+    mask[1] = 0                                     # a layer with nothing retained
+    sum_r = int(mask.sum())
+    # request-major dense states with padding between layers and requests
+    layer_stride = n_l * unit_words + 16
+    req_stride = L * layer_stride + 8
+    state = _state_with_specials(rng, (n_req * req_stride,))
+    pool = np.full((n_slots, sum_r * unit_words), np.float32(7.0))
+    src_req = np.array([2, 0, 3], np.int32)
+    dst_slot = np.array([5, 1, 2], np.int32)
+    oracle.pack(mask, unit_words, state, layer_stride, req_stride, src_req, pool, sum_r * unit_words, dst_slot)
+    bits = state.view(np.uint32)
+    for req, slot in zip(src_req, dst_slot):
+        dense = np.stack([bits[req * req_stride + l * layer_stride:][: n_l * unit_words].reshape(n_l, unit_words)
+                          for l in range(L)])
+        want = dense[mask.astype(bool)]             # layers ascending, units ascending
+        np.testing.assert_array_equal(pool[slot].view(np.uint32).reshape(sum_r, unit_words), want)
+    for slot in (0, 3, 4):                          # untouched slots
+        assert np.all(pool[slot] == np.float32(7.0))
+
+    out = np.full_like(state, np.float32(-3.0))
+    dst_req = np.array([1, 3, 0], np.int32)
+    oracle.restore(mask, unit_words, pool, sum_r * unit_words, dst_slot, out, layer_stride, req_stride, dst_req)
+    ob = out.view(np.uint32)
+    for src, dst in zip(src_req, dst_req):
+        for l in range(L):
+            a = bits[src * req_stride + l * layer_stride:][: n_l * unit_words].reshape(n_l, unit_words)
+            b = ob[dst * req_stride + l * layer_stride:][: n_l * unit_words].reshape(n_l, unit_words)
+            want = np.where(mask[l][:, None].astype(bool), a, np.uint32(0))   # masking, +0.0 bits
+            np.testing.assert_array_equal(b, want)
+            # padding after the layer is not written
+            pad = ob[dst * req_stride + l * layer_stride + n_l * unit_words:][:16]
+            assert np.all(pad.view(np.float32) == np.float32(-3.0))
+    # request 2 was no destination
+    assert np.all(out[2 * req_stride: 3 * req_stride] == np.float32(-3.0))
+
+
+def test_round_trip_all_retained_is_bit_exact():
+    rng = np.random.default_rng(6)
+    L, n_l, uw = 2, 12, 16
+    mask = np.ones((L, n_l), np.uint8)
+    state = _state_with_specials(rng, (3, L, n_l, uw))
+    pool = np.zeros((3, L * n_l * uw), np.float32)
+    ids = np.arange(3, dtype=np.int32)
+    oracle.pack(mask, uw, state, n_l * uw, L * n_l * uw, ids, pool, L * n_l * uw, ids[::-1].copy())
+    out = np.zeros_like(state)
+    oracle.restore(mask, uw, pool, L * n_l * uw, ids[::-1].copy(), out, n_l * uw, L * n_l * uw, ids)
+    np.testing.assert_array_equal(out.view(np.uint32), state.view(np.uint32))
+
+
+# ----------------------------------------------------------------------------
+# Eq. 1: the recurrence
+# ----------------------------------------------------------------------------
+
+def _run(kind, S0, q, k, v, g, beta, H_k=None, **kw):
+    """One layer, one request; S0 [H_v, d_k, d_v] fp32; streams [T, H, d]."""
+    H_v, d_k, d_v = S0.shape
+    H_k = H_k or H_v
+    T = q.shape[0]
+    state = S0.copy()
+    o, s64 = oracle.refresh(kind, 1, H_v, H_k, d_k, d_v, state, H_v * d_k * d_v, H_v * d_k * d_v, [0],
+                            np.ascontiguousarray(q, np.float32), np.ascontiguousarray(k, np.float32),
+                            np.ascontiguousarray(v, np.float32), np.ascontiguousarray(g, np.float32),
+                            np.ascontiguousarray(beta, np.float32), [0, T], want_state64=True, **kw)
+    return state, (o[0] if o is not None else None), s64[0, 0]
+
+
+def test_recurrence_beta_zero_is_pure_decay():
+    rng = np.random.default_rng(7)
+    T, H, dk, dv = 9, 2, 6, 5
+    S0 = rng.normal(size=(H, dk, dv)).astype(np.float32)
+    g = -rng.uniform(0.01, 1.0, size=(T, H, dk)).astype(np.float32)
+    k = rng.normal(size=(T, H, dk)); q = rng.normal(size=(T, H, dk)); v = rng.normal(size=(T, H, dv))
+    _, o, s64 = _run(oracle.KDA, S0, q, k, v, g, np.zeros((T, H), np.float32))
+    want = np.exp(g.astype(np.float64).sum(0))[:, :, None] * S0       # Diag(prod alpha) S_0 on the key index
+    np.testing.assert_allclose(s64, want, rtol=1e-13)
+    # read-out of a purely decaying state
+    qf = q.astype(np.float32).astype(np.float64)
+    St = np.exp(np.cumsum(g.astype(np.float64), 0))[:, :, :, None] * S0[None]
+    np.testing.assert_allclose(o, np.einsum("thc,thcv->thv", qf, St), rtol=1e-12, atol=1e-14)
+
+
+def test_recurrence_single_token_stores_value_at_key():
+    rng = np.random.default_rng(8)
+    dk, dv = 7, 4
+    k = rng.normal(size=(1, 1, dk)).astype(np.float32)
+    v = rng.normal(size=(1, 1, dv)).astype(np.float32)
+    S0 = rng.normal(size=(1, dk, dv)).astype(np.float32)
+    kk = k.astype(np.float64)
+    kk /= np.linalg.norm(kk)
+    # alpha = 1, beta = 1, |k| = 1 (up to fp32 rounding of k): S_1^T k = v
+    k32 = kk.astype(np.float32)
+    _, o, s64 = _run(oracle.KDA, S0, k32, k32, v, np.zeros((1, 1, dk), np.float32), np.ones((1, 1), np.float32))
+    n2 = float((k32.astype(np.float64) ** 2).sum())
+    read = s64[0].T @ k32[0, 0].astype(np.float64)
+    old = S0[0].astype(np.float64).T @ k32[0, 0].astype(np.float64)
+    # exact algebra with |k|^2 = n2: S^T k = old + n2 (v - old)
+    np.testing.assert_allclose(read, old + n2 * (v[0, 0] - old), rtol=1e-13)
+    np.testing.assert_allclose(read, v[0, 0], rtol=1e-6)
+    np.testing.assert_allclose(o[0, 0], read, rtol=1e-13)              # q = k reads it back
+
+
+def test_recurrence_one_hot_keys_pin_key_channel_decay():
+    # k_t = e_{pi(t)}: rows evolve independently as scalar AR(1) processes;
+    # row j sees alpha_{t,j} -- the decay is indexed by the KEY channel.
+    rng = np.random.default_rng(9)
+    T, dk, dv = 12, 5, 3
+    pi = rng.integers(0, dk, size=T)
+    k = np.zeros((T, 1, dk), np.float32)
+    k[np.arange(T), 0, pi] = 1.0
+    v = rng.normal(size=(T, 1, dv)).astype(np.float32)
+    g = -rng.uniform(0.05, 2.0, size=(T, 1, dk)).astype(np.float32)
+    beta = rng.uniform(0.1, 0.9, size=(T, 1)).astype(np.float32)
+    S0 = rng.normal(size=(1, dk, dv)).astype(np.float32)
+    q = rng.normal(size=(T, 1, dk)).astype(np.float32)
+    _, o, s64 = _run(oracle.KDA, S0, q, k, v, g, beta)
+    rows = S0[0].astype(np.float64).copy()
+    for t in range(T):
+        for j in range(dk):
+            a = math.exp(float(g[t, 0, j]))
+            if pi[t] == j:
+                rows[j] = (1.0 - float(beta[t, 0])) * a * rows[j] + float(beta[t, 0]) * v[t, 0].astype(np.float64)
+            else:
+                rows[j] = a * rows[j]
+        np.testing.assert_allclose(o[t, 0], rows.T @ q[t, 0].astype(np.float64), rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(s64[0], rows, rtol=1e-13)
+
+
+def test_recurrence_orthonormal_keys_scalar_decay_closed_form():
+    rng = np.random.default_rng(10)
+    T, dk, dv = 6, 8, 5
+    Q, _ = np.linalg.qr(rng.normal(size=(dk, dk)))
+    k = Q[:T].astype(np.float32)[:, None, :]                   # nearly orthonormal after fp32 rounding
+    v = rng.normal(size=(T, 1, dv)).astype(np.float32)
+    g = -rng.uniform(0.05, 0.7, size=(T, 1)).astype(np.float32)
+    beta = rng.uniform(0.1, 0.9, size=(T, 1)).astype(np.float32)
+    S0 = np.zeros((1, dk, dv), np.float32)
+    _, _, s64 = _run(oracle.GDN, S0, k, k, v, g, beta)
+    G = np.cumsum(g[:, 0].astype(np.float64))
+    want = np.zeros((dk, dv))
+    for i in range(T):
+        want += math.exp(G[-1] - G[i]) * float(beta[i, 0]) * np.outer(k[i, 0].astype(np.float64), v[i, 0].astype(np.float64))
+    # equality holds up to the fp32 rounding of the keys (k_i . k_j ~ 1e-7 for i != j)
+    np.testing.assert_allclose(s64[0], want, atol=5e-6)
+
+
+def test_gdn_equals_kda_with_broadcast_decay_and_grouped_heads():
+    rng = np.random.default_rng(11)
+    T, Hv, Hk, dk, dv = 10, 4, 2, 6, 5
+    S0 = rng.normal(size=(Hv, dk, dv)).astype(np.float32)
+    q = rng.normal(size=(T, Hk, dk)).astype(np.float32)
+    k = (rng.normal(size=(T, Hk, dk)) / 2).astype(np.float32)
+    v = rng.normal(size=(T, Hv, dv)).astype(np.float32)
+    g = -rng.uniform(0.01, 1.0, size=(T, Hv)).astype(np.float32)
+    beta = rng.uniform(0.1, 0.9, size=(T, Hv)).astype(np.float32)
+    s_g, o_g, _ = _run(oracle.GDN, S0, q, k, v, g, beta, H_k=Hk)
+    # KDA with one key head per value head (value head h reads key head h // 2) and g broadcast over channels
+    qq = np.repeat(q, Hv // Hk, axis=1); kk = np.repeat(k, Hv // Hk, axis=1)
+    s_k, o_k, _ = _run(oracle.KDA, S0, qq, kk, v, np.repeat(g[:, :, None], dk, axis=2), beta)
+    np.testing.assert_array_equal(s_g, s_k)
+    np.testing.assert_array_equal(o_g, o_k)
+
+
+def test_value_columns_are_independent():
+    rng = np.random.default_rng(12)
+    T, H, dk, dv = 8, 1, 6, 7
+    S0 = rng.normal(size=(H, dk, dv)).astype(np.float32)
+    q = rng.normal(size=(T, H, dk)).astype(np.float32); k = (rng.normal(size=(T, H, dk)) / 2).astype(np.float32)
+    v = rng.normal(size=(T, H, dv)).astype(np.float32)
+    g = -rng.uniform(0.01, 1.0, size=(T, H, dk)).astype(np.float32)
+    beta = rng.uniform(0.1, 0.9, size=(T, H)).astype(np.float32)
+    s_all, o_all, _ = _run(oracle.KDA, S0, q, k, v, g, beta)
+    perm = np.array([4, 0, 6])
+    s_sub, o_sub, _ = _run(oracle.KDA, np.ascontiguousarray(S0[:, :, perm]), q, k, np.ascontiguousarray(v[:, :, perm]), g, beta)
+    np.testing.assert_array_equal(s_sub, s_all[:, :, perm])
+    np.testing.assert_array_equal(o_sub, o_all[:, :, perm])
+
+
+def _chunk_form(S0, q, k, v, g, beta):
+    """Second formulation of Eq. 1 over a window: the deltas u_t solve a unit
+    lower-triangular system.  fp64 numpy + a library triangular solve."""
+    q, k, v, g, beta, S0 = (x.astype(np.float64) for x in (q, k, v, g, beta, S0))
+    G = np.cumsum(g, axis=0)
+    Kt, Kh, Qt = k * np.exp(G), k * np.exp(-G), q * np.exp(G)
+    A = np.tril(Kt @ Kh.T, -1) * beta[:, None]
+    U = scipy.linalg.solve_triangular(np.eye(len(beta)) + A, beta[:, None] * (v - Kt @ S0), lower=True,
+                                      unit_diagonal=True)
+    O = Qt @ S0 + np.tril(Qt @ Kh.T) @ U
+    S = np.exp(G[-1])[:, None] * (S0 + Kh.T @ U)
+    return S, O
+
+
+def test_chunk_identity_against_triangular_solve():
+    rng = np.random.default_rng(13)
+    T, dk, dv = 24, 16, 12
+    S0 = rng.normal(size=(1, dk, dv)).astype(np.float32)
+    q = rng.normal(size=(T, 1, dk)).astype(np.float32)
+    k = rng.normal(size=(T, 1, dk)); k = (k / np.linalg.norm(k, axis=-1, keepdims=True)).astype(np.float32)
+    v = rng.normal(size=(T, 1, dv)).astype(np.float32)
+    g = -rng.uniform(0.001, 0.5, size=(T, 1, dk)).astype(np.float32)
+    beta = rng.uniform(0.05, 0.95, size=(T, 1)).astype(np.float32)
+    _, o, s64 = _run(oracle.KDA, S0, q, k, v, g, beta)
+    S, O = _chunk_form(S0[0], q[:, 0], k[:, 0], v[:, 0], g[:, 0], beta[:, 0])
+    np.testing.assert_allclose(s64[0], S, rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(o[:, 0], O, rtol=1e-10, atol=1e-12)
+    # q_scale multiplies the outputs and nothing else
+    s2, o2, _ = _run(oracle.KDA, S0, q, k, v, g, beta, q_scale=0.25)
+    np.testing.assert_allclose(o2, 0.25 * o, rtol=1e-15)
+
+
+def test_bf16_streams_are_widened_exactly():
+    rng = np.random.default_rng(14)
+    T, H, dk, dv = 5, 2, 4, 3
+    # values already representable in bf16
+    def bf(x):
+        b = (x.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+        return b, (b.astype(np.uint32) << 16).view(np.float32)
+    qb, qf = bf(rng.normal(size=(1, T, H, dk))); kb, kf = bf(rng.normal(size=(1, T, H, dk)) / 2)
+    vb, vf = bf(rng.normal(size=(1, T, H, dv)))
+    g = -rng.uniform(0.01, 1.0, size=(1, T, H, dk)).astype(np.float32)
+    beta = rng.uniform(0.1, 0.9, size=(1, T, H)).astype(np.float32)
+    S0 = rng.normal(size=(H, dk, dv)).astype(np.float32)
+    sa = S0.copy(); sb = S0.copy()
+    oa, _ = oracle.refresh(oracle.KDA, 1, H, H, dk, dv, sa, H * dk * dv, H * dk * dv, [0], qb, kb, vb, g, beta, [0, T])
+    ob, _ = oracle.refresh(oracle.KDA, 1, H, H, dk, dv, sb, H * dk * dv, H * dk * dv, [0], qf, kf, vf, g, beta, [0, T])
+    np.testing.assert_array_equal(sa, sb)
+    np.testing.assert_array_equal(oa, ob)
+
+
+# ----------------------------------------------------------------------------
+# Composition invariants: checkpoint -> restore -> refresh
+# ----------------------------------------------------------------------------
+
+def _tiny_config(seed=0, L=2, H=4, d=8, T=48, n_req=3, rate=None):
+    rng = np.random.default_rng(seed)
+    rates = np.exp(rng.uniform(math.log(1e-3), 0.0, size=(L, H, d))).astype(np.float32)
+    if rate is not None:
+        rates[:] = rate
+    q = rng.normal(size=(L, T * n_req, H, d)); q = (q / np.linalg.norm(q, axis=-1, keepdims=True)).astype(np.float32)
+    k = rng.normal(size=(L, T * n_req, H, d)); k = (k / np.linalg.norm(k, axis=-1, keepdims=True)).astype(np.float32)
+    v = rng.normal(size=(L, T * n_req, H, d)).astype(np.float32)
+    g = (-np.log1p(np.exp(rng.normal(size=(L, T * n_req, H, d)))) * rates[:, None]).astype(np.float32)
+    beta = (1 / (1 + np.exp(-rng.normal(size=(L, T * n_req, H))))).astype(np.float32)
+    return rates, q, k, v, g, beta
+
+
+def _slice_tokens(x, n_req, T, lo, hi):
+    """Per-request token window [lo, hi) of streams laid out request after request."""
+    L = x.shape[0]
+    parts = [x[:, r * T + lo: r * T + hi] for r in range(n_req)]
+    return np.ascontiguousarray(np.concatenate(parts, axis=1))
+
+
+def test_full_prefix_replay_from_zero_equals_recomputation_and_continuation_is_exact():
+    L, H, d, T, n_req = 2, 4, 8, 48, 3
+    rates, q, k, v, g, beta = _tiny_config(0, L, H, d, T, n_req)
+    ls, rs = H * d * d, L * H * d * d
+    ids = np.arange(n_req, dtype=np.int32)
+    cu_full = np.arange(n_req + 1, dtype=np.int32) * T
+    # uninterrupted run over the whole prefix from a zero state
+    full = np.zeros((n_req, L, H, d, d), np.float32)
+    o_full, s64_full = oracle.refresh(oracle.KDA, L, H, H, d, d, full, ls, rs, ids, q, k, v, g, beta, cu_full,
+                                      want_state64=True)
+    # the same thing written as one unit at a time (harness slicing / cu_seqlens check)
+    for r in (0, 2):
+        for l in (0, 1):
+            one = np.zeros((H, d, d), np.float32)
+            sl = slice(r * T, (r + 1) * T)
+            o1, _ = oracle.refresh(oracle.KDA, 1, H, H, d, d, one, ls, ls, [0], np.ascontiguousarray(q[l:l + 1, sl]),
+                                   np.ascontiguousarray(k[l:l + 1, sl]), np.ascontiguousarray(v[l:l + 1, sl]),
+                                   np.ascontiguousarray(g[l:l + 1, sl]), np.ascontiguousarray(beta[l:l + 1, sl]), [0, T])
+            np.testing.assert_array_equal(one, full[r, l])
+            np.testing.assert_array_equal(o1[0], o_full[l, sl])
+    # checkpoint at p, keep everything, restore, continue over (p, T]: identical in fp64 to the uninterrupted run
+    p = 32
+    cu_a = np.arange(n_req + 1, dtype=np.int32) * p
+    cu_b = np.arange(n_req + 1, dtype=np.int32) * (T - p)
+    part = np.zeros((n_req, L, H, d, d), np.float32)
+    head = [_slice_tokens(x, n_req, T, 0, p) for x in (q, k, v, g, beta)]
+    tail = [_slice_tokens(x, n_req, T, p, T) for x in (q, k, v, g, beta)]
+    _, s64_p = oracle.refresh(oracle.KDA, L, H, H, d, d, part, ls, rs, ids, *head, cu_a, want_state64=True)
+    mask = np.ones((L, H * d), np.uint8)
+    pool = np.zeros((n_req, L * H * d * d), np.float32)
+    oracle.pack(mask, d, part, ls, rs, ids, pool, L * H * d * d, ids)
+    back = np.full_like(part, 9.0)
+    oracle.restore(mask, d, pool, L * H * d * d, ids, back, ls, rs, ids)
+    np.testing.assert_array_equal(back, part)
+    o_tail, s64_tail = oracle.refresh(oracle.KDA, L, H, H, d, d, back, ls, rs, ids, *tail, cu_b, want_state64=True)
+    # the checkpoint rounds the state to fp32 once; beyond that the run is the same operation sequence
+    np.testing.assert_allclose(s64_tail, s64_full, rtol=2e-6, atol=2e-7)
+    for r in range(n_req):
+        np.testing.assert_allclose(o_tail[:, r * (T - p):(r + 1) * (T - p)], o_full[:, r * T + p:(r + 1) * T],
+                                   rtol=2e-6, atol=2e-7)
+
+
+def test_scratch_merge_local_writes_only_omitted_units():
+    L, H, d, T, n_req = 2, 4, 8, 48, 3
+    rates, q, k, v, g, beta = _tiny_config(1, L, H, d, T, n_req)
+    ls, rs = H * d * d, L * H * d * d
+    ids = np.arange(n_req, dtype=np.int32)
+    A_log = np.log(rates).reshape(L, H * d)
+    plan = oracle.plan(oracle.KDA, L, H, d, A_log, np.zeros_like(A_log), sel=oracle.SEL_TOP_RATIO, keep_ratio=0.4,
+                       scope=oracle.SCOPE_HEAD)
+    rng = np.random.default_rng(2)
+    stored = rng.normal(size=(n_req, L, H, d, d)).astype(np.float32)
+    W = 16
+    tail = [_slice_tokens(x, n_req, T, T - W, T) for x in (q, k, v, g, beta)]
+    cu = np.arange(n_req + 1, dtype=np.int32) * W
+    merged = stored.copy()
+    oracle.refresh(oracle.KDA, L, H, H, d, d, merged, ls, rs, ids, *tail, cu, want_o=False,
+                   mode=oracle.MODE_SCRATCH_MERGE_LOCAL, mask=plan.mask)
+    scratch = np.zeros_like(stored)
+    oracle.refresh(oracle.KDA, L, H, H, d, d, scratch, ls, rs, ids, *tail, cu, want_o=False)
+    keep = plan.mask.reshape(L, H, d).astype(bool)[None, :, :, :, None]
+    np.testing.assert_array_equal(merged, np.where(keep, stored, scratch))
+    # GDN: whole heads
+    gmask = np.array([[1, 0, 0, 1], [0, 1, 1, 0]], np.uint8)
+    gg = np.ascontiguousarray(tail[3][..., 0])
+    merged = stored.copy()
+    oracle.refresh(oracle.GDN, L, H, H, d, d, merged, ls, rs, ids, tail[0], tail[1], tail[2], gg, tail[4], cu,
+                   want_o=False, mode=oracle.MODE_SCRATCH_MERGE_LOCAL, mask=gmask)
+    scratch = np.zeros_like(stored)
+    oracle.refresh(oracle.GDN, L, H, H, d, d, scratch, ls, rs, ids, tail[0], tail[1], tail[2], gg, tail[4], cu, want_o=False)
+    np.testing.assert_array_equal(merged, np.where(gmask.astype(bool)[None, :, :, None, None], stored, scratch))
+
+
+def test_zero_fill_refresh_error_shrinks_with_window():
+    # Section 4.2: the suffix refresh is approximate because history before the window is lost;
+    # short-horizon (omitted) rows forget that history quickly, so a longer window can only help.
+    L, H, d, T, n_req = 1, 2, 8, 96, 1
+    rates, q, k, v, g, beta = _tiny_config(3, L, H, d, T, n_req, rate=1.0)   # every unit short-horizon
+    ls = H * d * d
+    truth = np.zeros((1, L, H, d, d), np.float32)
+    oracle.refresh(oracle.KDA, L, H, H, d, d, truth, ls, ls, [0], q, k, v, g, beta, [0, T], want_o=False)
+    errs = []
+    for W in (4, 16, 64):
+        tail = [np.ascontiguousarray(x[:, T - W:]) for x in (q, k, v, g, beta)]
+        s = np.zeros_like(truth)
+        oracle.refresh(oracle.KDA, L, H, H, d, d, s, ls, ls, [0], *tail, [0, W], want_o=False,
+                       mode=oracle.MODE_SCRATCH_MERGE_LOCAL, mask=np.zeros((L, H * d), np.uint8))
+        errs.append(np.abs(s - truth).max())
+    assert errs[0] > errs[1] > errs[2]
+    assert errs[2] < 1e-6
+
+
+# ----------------------------------------------------------------------------
+# Appendix D: INT8 quantiser
+# ----------------------------------------------------------------------------
+
+def test_int8_quantiser_properties():
+    rng = np.random.default_rng(15)
+    rows = rng.normal(size=(6, 32)).astype(np.float32)
+    rows[1] = 0.0                                            # all-zero row: scale floor 1e-8/127
+    rows[2, 3] = 50.0
+    rows[3] = np.arange(32, dtype=np.float32) - 16           # hand-checkable
+    q, s = oracle.int8_quantize(rows)
+    assert s.dtype == np.float32 and q.dtype == np.int8
+    assert s[1] == np.float32(1e-8) / np.float32(127) and np.all(q[1] == 0)
+    assert np.all(np.abs(q) <= 127)
+    amax = np.abs(rows).max(1)
+    np.testing.assert_array_equal(s[[0, 2, 3, 4, 5]], (amax / np.float32(127))[[0, 2, 3, 4, 5]])
+    # the largest magnitude of each row maps to +-127
+    for r in (0, 2, 3, 4, 5):
+        assert np.abs(q[r]).max() == 127
+    # row 3: scale = 16/127, q = round(x * 127/16): ties-to-even on exact halves
+    want = np.array([np.float32(x) / s[3] for x in rows[3]], np.float32)
+    np.testing.assert_array_equal(q[3], np.rint(want).astype(np.int8))
+    back = oracle.int8_dequantize(q, s)
+    assert np.all(np.abs(back - rows) <= 0.5 * s[:, None] * (1 + 1e-6))
+    # ties to even: 0.5*s -> 0, 1.5*s -> 2, 2.5*s -> 2
+    t = np.zeros((1, 4), np.float32); t[0] = [127.0, 0.5, 1.5, 2.5]
+    qq, ss = oracle.int8_quantize(t)
+    assert ss[0] == 1.0 and list(qq[0]) == [127, 0, 2, 2]
