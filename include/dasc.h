@@ -1,0 +1,247 @@
+/*
+ * dasc.h -- C ABI of the B200 (sm_100a) implementation of the data-parallel
+ * hot path of Decay-Aware State Compression (DASC): the compress / restore
+ * cycle of linear-attention recurrent-state checkpoints in a prefix cache.
+ *
+ *   dasc_plan     host   static selection plan          (Section 3.3, 4.1, Eq. 2/3/6/7, App. B)
+ *   dasc_pack     device retained units -> ragged pool  (Store path, Section 4.1, App. B Scheme 2)
+ *   dasc_restore  device pool -> dense state, zero-fill (Load path, zero-fill policy, Section 4.2)
+ *   dasc_refresh  device replay of the gated delta rule (Eq. 1; suffix-refresh policy, Section 4.2)
+ *
+ * Conventions
+ *   - No exception crosses this boundary; every call returns a dasc_status_t.
+ *   - "HOST" / "DEVICE" on a pointer says where the memory lives.  All device
+ *     buffers are owned by the caller; the library owns only the plan object
+ *     and the small index tables it uploads once in dasc_plan.
+ *   - Device calls are asynchronous on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream), never synchronise, never
+ *     allocate, and may be issued concurrently on several streams against one
+ *     plan (a plan is immutable after creation).
+ *   - Argument errors are detected on the host before any launch and leave
+ *     the outputs untouched.
+ *   - State orientation: the paper writes the recurrent state as S in
+ *     R^{d_v x d_k} with o = S q (Section 3.1).  This library stores the
+ *     transpose, S[head][d_k][d_v], fp32, row-major, so that one KDA key
+ *     channel S_{h,:,k} (the KDA selection unit of Section 4.1) is one
+ *     contiguous row of d_v floats.  A dense state is addressed as
+ *         state_base + req*req_stride + layer*layer_stride
+ *                    + ((head*d_k + k)*d_v + v)            [floats]
+ *     so both layer-major and request-major active-state pools work.
+ *   - Selection units (Section 4.1): KDA -> one (head, key channel) row of
+ *     d_v floats; GDN -> one complete value-head state of d_k*d_v floats.
+ *     Unit index inside a layer: u = head*d_k + k (KDA), u = head (GDN).
+ *   - Checkpoint pool (Appendix B, ragged layout): slot s holds, for layers
+ *     in ascending order, the retained units of that layer in ascending unit
+ *     index; layer l occupies units [o_l, o_{l+1}) with o_0 = 0 and
+ *     o_{l+1} = o_l + r_l.  Slot s starts at pool_base + s*slot_stride floats.
+ */
+#ifndef DASC_H_
+#define DASC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DASC_OK = 0,
+  DASC_ERR_INVALID_ARG = 1, /* null pointer, negative size, misaligned pointer or stride */
+  DASC_ERR_SHAPE = 2,       /* shape outside what the kernels support */
+  DASC_ERR_UNSUPPORTED = 3, /* valid request that this build does not implement */
+  DASC_ERR_ALLOC = 4,       /* host or device allocation failed (dasc_plan only) */
+  DASC_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed */
+  DASC_ERR_WORKSPACE = 6,   /* workspace missing, misaligned or too small */
+  DASC_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (reported by dasc_refresh_status) */
+} dasc_status_t;
+
+typedef enum { DASC_KDA = 0, DASC_GDN = 1 } dasc_kind_t;
+typedef enum {
+  DASC_SEL_THRESHOLD = 0, /* retained iff H_s > w_max, strictly (Section 4.1) */
+  DASC_SEL_TOP_RATIO = 1, /* keep the ceil(keep_ratio*n) longest-horizon units of each scope group */
+  DASC_SEL_EXPLICIT = 2   /* caller-supplied mask */
+} dasc_sel_t;
+typedef enum { DASC_SCOPE_HEAD = 0, DASC_SCOPE_LAYER = 1, DASC_SCOPE_MODEL = 2 } dasc_scope_t;
+typedef enum { DASC_IO_BF16 = 0, DASC_IO_FP32 = 1 } dasc_io_dtype_t;
+typedef enum {
+  DASC_REFRESH_CONTINUE = 0,           /* start from the stored state, write every unit back */
+  DASC_REFRESH_SCRATCH_MERGE_LOCAL = 1 /* start from zero, write back only the omitted units */
+} dasc_refresh_mode_t;
+typedef enum {
+  DASC_ALGO_AUTO = 0,
+  DASC_ALGO_SEQUENTIAL = 1, /* token-by-token fp32 kernel; any log-decay */
+  DASC_ALGO_CHUNKED = 2     /* chunked (UT-transform) tensor-core kernel; see dasc_refresh */
+} dasc_refresh_algo_t;
+
+typedef struct dasc_plan_s dasc_plan_t; /* opaque */
+
+/*
+ * Plan description.  All pointers are HOST memory and are only read during
+ * dasc_plan.  A_log and dt_bias hold one entry per selection unit, laid out
+ * [n_layers][n_v_heads][units_per_head] with units_per_head = d_k (KDA) or
+ * 1 (GDN); a caller whose model has one parameter per head broadcasts it.
+ */
+typedef struct {
+  int32_t kind;                 /* dasc_kind_t */
+  int32_t n_layers;             /* recurrent (linear-attention) layers only */
+  int32_t n_v_heads;            /* value heads = number of head states per layer */
+  int32_t n_k_heads;            /* key/query heads; divides n_v_heads; value head h reads key head h/(n_v_heads/n_k_heads) */
+  int32_t d_k, d_v;             /* d_v must be a multiple of 4 (16-byte rows) */
+  const float *A_log;           /* HOST, Eq. 2 */
+  const float *dt_bias;         /* HOST, Eq. 2 */
+  double a;                     /* fixed gate logit of the static metric; the paper uses -0.3 */
+  double eps;                   /* Eq. 3; the paper uses 1e-3 */
+  int32_t sel;                  /* dasc_sel_t */
+  int32_t scope;                /* dasc_scope_t; TOP_RATIO only */
+  double w_max;                 /* threshold of Section 4.1 and window cap of Eq. 7.  With TOP_RATIO or
+                                   EXPLICIT, w_max <= 0 means: cap = next power of two of the largest
+                                   omitted horizon. */
+  double keep_ratio;            /* TOP_RATIO only, in [0, 1] */
+  int32_t randomize;            /* != 0: replace each layer's selection by a seeded uniform draw of the
+                                   same count r_l (the count-matched random control of Appendix C.3) */
+  uint64_t seed;                /* for randomize */
+  const uint8_t *explicit_mask; /* HOST, EXPLICIT only: [n_layers][units per layer], != 0 = retained */
+  int64_t conv_bytes_per_ckpt;  /* B_conv of Eq. 6 (uncompressed convolution state), may be 0 */
+} dasc_plan_desc_t;
+
+/* Scalar results of a plan (Eq. 6, Eq. 7, Appendix B). */
+typedef struct {
+  int32_t kind, n_layers, n_v_heads, n_k_heads, d_k, d_v;
+  int64_t units_per_layer;   /* n_l */
+  int64_t unit_floats;       /* d_v (KDA) or d_k*d_v (GDN) */
+  int64_t units_total;       /* sum_l n_l */
+  int64_t units_retained;    /* sum_l r_l */
+  int64_t r_max;             /* max_l r_l */
+  int64_t slot_floats;       /* units_retained * unit_floats: the compact slot stride */
+  int64_t dense_floats_per_layer; /* n_v_heads*d_k*d_v */
+  double c_temp_rag;         /* Eq. 6: sum n_l / sum r_l        (inf if nothing is retained) */
+  double c_temp_pad;         /* App. B: sum n_l / (L * R_max)   (inf if nothing is retained) */
+  double c_ckpt_rag;         /* Eq. 6: (B_dense + B_conv) / (B_rag + B_conv) */
+  double w_max_used;         /* window cap used by Eq. 7 */
+  int64_t w_replay;          /* Eq. 7: max over omitted units of W_u; 0 if nothing is omitted */
+  int32_t device;            /* CUDA device holding the index tables, -1 for a host-only plan */
+} dasc_plan_info_t;
+
+/*
+ * Build the static selection plan (Section 4.1; it depends on model weights only,
+ * so it is built once, before serving).
+ * For every unit: g = -exp(A_log) * softplus(a + dt_bias) (Eq. 2),
+ * H_s = ln(eps)/g (Eq. 3), all in fp64.  Selection per `sel`; TOP_RATIO keeps,
+ * in each scope group of n units, the r = ceil(keep_ratio*n - 1e-9) units of
+ * largest H_s, ties to the lower unit index.  Replay windows per Eq. 7:
+ * W_u = clamp(next_pow2(H_s(u)), 4, w_max) with next_pow2 the smallest power
+ * of two >= H_s, W_replay = max over omitted units.
+ *
+ * device >= 0: also uploads the index tables pack/restore/refresh need to
+ * that CUDA device (the only device allocation this library ever makes).
+ * device  < 0: host-only plan; the accessors work, device calls return
+ * DASC_ERR_INVALID_ARG.
+ * On error *out is NULL.
+ */
+dasc_status_t dasc_plan(const dasc_plan_desc_t *desc, int32_t device, dasc_plan_t **out);
+void dasc_plan_destroy(dasc_plan_t *plan);
+
+/* Accessors.  Array outputs are HOST buffers the caller sized from dasc_plan_info:
+ * horizon/mask/window: n_layers*units_per_layer entries, [layer][unit];
+ * layer_counts: n_layers (r_l); layer_offsets: n_layers+1 (o_l). */
+dasc_status_t dasc_plan_info(const dasc_plan_t *plan, dasc_plan_info_t *out);
+dasc_status_t dasc_plan_horizon(const dasc_plan_t *plan, double *out);
+dasc_status_t dasc_plan_mask(const dasc_plan_t *plan, uint8_t *out);
+dasc_status_t dasc_plan_window(const dasc_plan_t *plan, int64_t *out);
+dasc_status_t dasc_plan_layer_counts(const dasc_plan_t *plan, int64_t *out);
+dasc_status_t dasc_plan_layer_offsets(const dasc_plan_t *plan, int64_t *out);
+
+/*
+ * Store path (Section 4.1; Appendix B, ragged layout): for each pair i,
+ *     pool[dst_slot[i]][o_l + j] = unit j-th retained of layer l of request src_req[i]
+ * as a bit copy (values are never interpreted; NaN payloads, -0.0 and
+ * denormals survive).
+ *   state_base  DEVICE, const, 16-byte aligned; strides in floats, multiples of 4.
+ *   src_req     DEVICE int32[n_pairs]: request index of each source state.
+ *   pool_base   DEVICE, 16-byte aligned.
+ *   slot_stride floats between slots, multiple of 4, >= slot_floats; 0 = slot_floats.
+ *   dst_slot    DEVICE int32[n_pairs]; destination slots must be distinct.
+ * n_pairs == 0 is a no-op.  Source and pool must not overlap.
+ */
+dasc_status_t dasc_pack(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride,
+                        int64_t req_stride, const int32_t *src_req, float *pool_base,
+                        int64_t slot_stride, const int32_t *dst_slot, int32_t n_pairs,
+                        void *cuda_stream);
+
+/*
+ * Load path, zero-fill policy (Section 4.2: retained units are loaded exactly,
+ * omitted units are left at zero).  For each pair i every float of the dense
+ * state of request dst_req[i] (all layers, all heads) is written exactly once:
+ * a retained unit gets the bits stored in slot src_slot[i], an omitted unit
+ * gets +0.0f (all-zero bits).  Memory between the dense layers (when
+ * layer_stride exceeds the dense layer size) is not touched.
+ * Pointer, alignment and stride rules as for dasc_pack; dst_req must be distinct.
+ */
+dasc_status_t dasc_restore(const dasc_plan_t *plan, const float *pool_base, int64_t slot_stride,
+                           const int32_t *src_slot, float *state_base, int64_t layer_stride,
+                           int64_t req_stride, const int32_t *dst_req, int32_t n_pairs,
+                           void *cuda_stream);
+
+/*
+ * Suffix refresh: replay the gated delta rule (Eq. 1, transposed orientation)
+ *     S_t = (I - beta_t k_t k_t^T) Diag(alpha_t) S_{t-1} + beta_t k_t v_t^T,   alpha_t = exp(g_t)
+ *     o_t = q_scale * S_t^T q_t
+ * over each request's token range, for layers [layer_begin, layer_end) and
+ * all value heads, updating the fp32 states in place.  alpha_t is channel-wise
+ * for KDA and one scalar per value head for GDN.
+ *
+ * Token streams (DEVICE, const), with Lc = layer_end - layer_begin and
+ * T = total_tokens = cu_seqlens[n_req]:
+ *   q, k   [Lc][T][n_k_heads][d_k]   bf16 or fp32 (io_dtype)
+ *   v      [Lc][T][n_v_heads][d_v]   same dtype
+ *   g      [Lc][T][n_v_heads][d_k]   fp32 log-decay, KDA;  [Lc][T][n_v_heads] for GDN
+ *   beta   [Lc][T][n_v_heads]        fp32
+ *   o      [Lc][T][n_v_heads][d_v]   o_dtype (bf16 or fp32, independent of io_dtype), out;
+ *                                     NULL = outputs not wanted
+ *   cu_seqlens DEVICE int32[n_req+1], ascending from 0: request r owns tokens
+ *          [cu_seqlens[r], cu_seqlens[r+1]) of every layer; empty ranges are allowed.
+ *   req_idx    DEVICE int32[n_req]: which dense state each request updates (distinct).
+ *   max_seqlen an upper bound on any request's token count (sizes the launch).
+ *
+ * mode CONTINUE: S_0 is the state as stored (for instance just restored);
+ *   every unit is written back.  This continues the recurrence.
+ * mode SCRATCH_MERGE_LOCAL (the paper's suffix-refresh load policy, Section 4.2):
+ *   S_0 = 0 in a scratch state; afterwards only the units the plan OMITS are
+ *   copied into the stored state, retained units keep their stored values.
+ *
+ * algo SEQUENTIAL is exact fp32 arithmetic token by token and accepts any g <= 0.
+ * algo CHUNKED processes 64-token chunks on the tensor cores; it needs
+ *   d_k = d_v = 128 and, for every 32 consecutive tokens and every channel,
+ *   sum |g| <= 80 (decay factors are formed relative to the chunk midpoint in
+ *   fp32).  AUTO picks CHUNKED when the shape allows it.
+ *
+ * workspace: DEVICE scratch of at least dasc_refresh_workspace_bytes(), 256-byte
+ *   aligned, private to this call until it completes; may be NULL when that
+ *   size is 0.
+ * Errors: bad arguments -> no launch.  A bounded device-side wait that runs
+ *   out sets a flag in the workspace; read it with dasc_refresh_status after
+ *   synchronising the stream.
+ */
+dasc_status_t dasc_refresh_workspace_bytes(const dasc_plan_t *plan, int32_t n_req, int32_t n_layers_in_call,
+                                           int32_t algo, size_t *out);
+dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t layer_stride,
+                           int64_t req_stride, const int32_t *req_idx, const void *q, const void *k,
+                           const void *v, int32_t io_dtype, const float *g, const float *beta,
+                           const int32_t *cu_seqlens, int32_t n_req, int64_t total_tokens,
+                           int32_t max_seqlen, int32_t layer_begin, int32_t layer_end, float q_scale,
+                           void *o, int32_t o_dtype, int32_t mode, int32_t algo, void *workspace,
+                           size_t workspace_bytes, void *cuda_stream);
+/* After the stream has been synchronised: DASC_OK, or DASC_ERR_TIMEOUT if a
+ * device-side wait of the last dasc_refresh that used `workspace` gave up.
+ * Copies 4 bytes device -> host (synchronous). */
+dasc_status_t dasc_refresh_status(const void *workspace, size_t workspace_bytes);
+
+const char *dasc_status_string(dasc_status_t status);
+/* "major.minor.patch" of this library. */
+const char *dasc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DASC_H_ */

@@ -1,0 +1,266 @@
+// C ABI of libdasc: argument validation and marshalling only; all work happens
+// in plan_host.cpp (host plan) and in the CUDA kernels.
+#include <cuda_runtime.h>
+
+#include <cstring>
+#include <new>
+
+#include "dasc_internal.h"
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+template <typename T>
+cudaError_t upload(T **dst, const T *src, size_t n) {
+  *dst = nullptr;
+  const size_t bytes = (n ? n : 1) * sizeof(T);
+  cudaError_t e = cudaMalloc(reinterpret_cast<void **>(dst), bytes);
+  if (e != cudaSuccess) return e;
+  if (n) e = cudaMemcpy(*dst, src, n * sizeof(T), cudaMemcpyHostToDevice);
+  return e;
+}
+
+void free_device_tables(dasc_plan_s *p) {
+  if (p->info.device < 0) return;
+  DeviceGuard guard(p->info.device);
+  cudaFree(p->d_row_src);
+  cudaFree(p->d_row_pos);
+  cudaFree(p->d_row_keep);
+  p->d_row_src = nullptr;
+  p->d_row_pos = nullptr;
+  p->d_row_keep = nullptr;
+}
+
+dasc_status_t check_copy_args(const dasc_plan_t *plan, const void *state, int64_t layer_stride, int64_t req_stride,
+                              const void *idx_a, const void *pool, int64_t *slot_stride, const void *idx_b,
+                              int32_t n_pairs) {
+  if (!plan) return DASC_ERR_INVALID_ARG;
+  if (plan->info.device < 0) return DASC_ERR_INVALID_ARG;
+  if (n_pairs < 0) return DASC_ERR_INVALID_ARG;
+  if (n_pairs == 0) return DASC_OK;
+  if (!state || !pool || !idx_a || !idx_b) return DASC_ERR_INVALID_ARG;
+  if (!aligned16(state) || !aligned16(pool)) return DASC_ERR_INVALID_ARG;
+  if (*slot_stride == 0) *slot_stride = plan->info.slot_floats;
+  if (layer_stride < 0 || req_stride < 0 || *slot_stride < plan->info.slot_floats) return DASC_ERR_INVALID_ARG;
+  if (layer_stride % 4 || req_stride % 4 || *slot_stride % 4) return DASC_ERR_INVALID_ARG;
+  if (plan->info.n_layers > 1 && layer_stride < plan->info.dense_floats_per_layer &&
+      req_stride < plan->info.dense_floats_per_layer)
+    return DASC_ERR_INVALID_ARG;  // layers of one request would overlap
+  // 32-bit vector indices inside the kernels
+  const int64_t vpr = plan->info.d_v / 4;
+  if (plan->packed_rows * vpr >= (int64_t{1} << 31) || plan->rows_per_layer * vpr >= (int64_t{1} << 31))
+    return DASC_ERR_SHAPE;
+  return DASC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+dasc_status_t dasc_plan(const dasc_plan_desc_t *desc, int32_t device, dasc_plan_t **out) {
+  if (!out) return DASC_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!desc) return DASC_ERR_INVALID_ARG;
+  dasc_plan_s *p = new (std::nothrow) dasc_plan_s();
+  if (!p) return DASC_ERR_ALLOC;
+  dasc_status_t st;
+  try {
+    st = dasc_build_plan_host(desc, p);
+  } catch (const std::bad_alloc &) {
+    st = DASC_ERR_ALLOC;
+  } catch (...) {
+    st = DASC_ERR_INVALID_ARG;
+  }
+  if (st != DASC_OK) {
+    delete p;
+    return st;
+  }
+  if (device >= 0) {
+    DeviceGuard guard(device);
+    if (!guard.ok) {
+      delete p;
+      return DASC_ERR_CUDA;
+    }
+    p->info.device = device;
+    std::vector<uint8_t> keep(p->row_pos.size());
+    for (size_t i = 0; i < keep.size(); ++i) keep[i] = p->row_pos[i] >= 0 ? 1 : 0;
+    cudaError_t e = upload(&p->d_row_src, p->row_src.data(), p->row_src.size());
+    if (e == cudaSuccess) e = upload(&p->d_row_pos, p->row_pos.data(), p->row_pos.size());
+    if (e == cudaSuccess) e = upload(&p->d_row_keep, keep.data(), keep.size());
+    if (e != cudaSuccess) {
+      free_device_tables(p);
+      delete p;
+      return e == cudaErrorMemoryAllocation ? DASC_ERR_ALLOC : DASC_ERR_CUDA;
+    }
+  }
+  *out = p;
+  return DASC_OK;
+}
+
+void dasc_plan_destroy(dasc_plan_t *plan) {
+  if (!plan) return;
+  free_device_tables(plan);
+  delete plan;
+}
+
+dasc_status_t dasc_plan_info(const dasc_plan_t *plan, dasc_plan_info_t *out) {
+  if (!plan || !out) return DASC_ERR_INVALID_ARG;
+  *out = plan->info;
+  return DASC_OK;
+}
+
+#define DASC_COPY_OUT(field)                                                        \
+  if (!plan || !out) return DASC_ERR_INVALID_ARG;                                   \
+  std::memcpy(out, plan->field.data(), plan->field.size() * sizeof(plan->field[0])); \
+  return DASC_OK;
+
+dasc_status_t dasc_plan_horizon(const dasc_plan_t *plan, double *out) { DASC_COPY_OUT(horizon) }
+dasc_status_t dasc_plan_mask(const dasc_plan_t *plan, uint8_t *out) { DASC_COPY_OUT(mask) }
+dasc_status_t dasc_plan_window(const dasc_plan_t *plan, int64_t *out) { DASC_COPY_OUT(window) }
+dasc_status_t dasc_plan_layer_counts(const dasc_plan_t *plan, int64_t *out) { DASC_COPY_OUT(layer_count) }
+dasc_status_t dasc_plan_layer_offsets(const dasc_plan_t *plan, int64_t *out) { DASC_COPY_OUT(layer_offset) }
+#undef DASC_COPY_OUT
+
+dasc_status_t dasc_pack(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride, int64_t req_stride,
+                        const int32_t *src_req, float *pool_base, int64_t slot_stride, const int32_t *dst_slot,
+                        int32_t n_pairs, void *cuda_stream) {
+  dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, src_req, pool_base, &slot_stride,
+                                     dst_slot, n_pairs);
+  if (st != DASC_OK || n_pairs == 0) return st;
+  const int e = dasc_launch_pack(plan, state_base, layer_stride, req_stride, src_req, pool_base, slot_stride,
+                                 dst_slot, n_pairs, cuda_stream);
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+dasc_status_t dasc_restore(const dasc_plan_t *plan, const float *pool_base, int64_t slot_stride,
+                           const int32_t *src_slot, float *state_base, int64_t layer_stride, int64_t req_stride,
+                           const int32_t *dst_req, int32_t n_pairs, void *cuda_stream) {
+  dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, dst_req, pool_base, &slot_stride,
+                                     src_slot, n_pairs);
+  if (st != DASC_OK || n_pairs == 0) return st;
+  const int e = dasc_launch_restore(plan, pool_base, slot_stride, src_slot, state_base, layer_stride, req_stride,
+                                    dst_req, n_pairs, cuda_stream);
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+static bool chunked_shape_ok(const dasc_plan_t *plan) { return plan->info.d_k == 128 && plan->info.d_v == 128; }
+
+dasc_status_t dasc_refresh_workspace_bytes(const dasc_plan_t *plan, int32_t n_req, int32_t n_layers_in_call,
+                                           int32_t algo, size_t *out) {
+  if (!plan || !out || n_req < 0 || n_layers_in_call < 0) return DASC_ERR_INVALID_ARG;
+  if (algo != DASC_ALGO_AUTO && algo != DASC_ALGO_SEQUENTIAL && algo != DASC_ALGO_CHUNKED) return DASC_ERR_INVALID_ARG;
+  const bool chunked = algo == DASC_ALGO_CHUNKED || (algo == DASC_ALGO_AUTO && chunked_shape_ok(plan));
+  *out = chunked ? dasc_refresh_chunked_workspace_bytes(n_req, n_layers_in_call, plan->info.n_v_heads) : 0;
+  return DASC_OK;
+}
+
+dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t layer_stride, int64_t req_stride,
+                           const int32_t *req_idx, const void *q, const void *k, const void *v, int32_t io_dtype,
+                           const float *g, const float *beta, const int32_t *cu_seqlens, int32_t n_req,
+                           int64_t total_tokens, int32_t max_seqlen, int32_t layer_begin, int32_t layer_end,
+                           float q_scale, void *o, int32_t o_dtype, int32_t mode, int32_t algo, void *workspace,
+                           size_t workspace_bytes, void *cuda_stream) {
+  if (!plan || plan->info.device < 0) return DASC_ERR_INVALID_ARG;
+  if (n_req < 0 || total_tokens < 0 || max_seqlen < 0) return DASC_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_end < layer_begin || layer_end > plan->info.n_layers) return DASC_ERR_INVALID_ARG;
+  if (io_dtype != DASC_IO_BF16 && io_dtype != DASC_IO_FP32) return DASC_ERR_INVALID_ARG;
+  if (o && o_dtype != DASC_IO_BF16 && o_dtype != DASC_IO_FP32) return DASC_ERR_INVALID_ARG;
+  if (mode != DASC_REFRESH_CONTINUE && mode != DASC_REFRESH_SCRATCH_MERGE_LOCAL) return DASC_ERR_INVALID_ARG;
+  if (algo != DASC_ALGO_AUTO && algo != DASC_ALGO_SEQUENTIAL && algo != DASC_ALGO_CHUNKED) return DASC_ERR_INVALID_ARG;
+  if (n_req == 0 || layer_end == layer_begin || total_tokens == 0) return DASC_OK;
+  if (!state_base || !req_idx || !q || !k || !v || !g || !beta || !cu_seqlens) return DASC_ERR_INVALID_ARG;
+  if (!aligned16(state_base) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) ||
+      (o && !aligned16(o)))
+    return DASC_ERR_INVALID_ARG;
+  if (layer_stride < 0 || req_stride < 0 || layer_stride % 4 || req_stride % 4) return DASC_ERR_INVALID_ARG;
+  const size_t esz = io_dtype == DASC_IO_BF16 ? 2 : 4;
+  if ((plan->info.d_k * esz) % 16 || (plan->info.d_v * esz) % 16) return DASC_ERR_SHAPE;
+
+  bool chunked = algo == DASC_ALGO_CHUNKED || (algo == DASC_ALGO_AUTO && chunked_shape_ok(plan));
+  if (algo == DASC_ALGO_CHUNKED && !chunked_shape_ok(plan)) return DASC_ERR_SHAPE;
+
+  DascRefreshArgs a{};
+  a.kind = plan->info.kind;
+  a.H_v = plan->info.n_v_heads;
+  a.H_k = plan->info.n_k_heads;
+  a.d_k = plan->info.d_k;
+  a.d_v = plan->info.d_v;
+  a.state = state_base;
+  a.layer_stride = layer_stride;
+  a.req_stride = req_stride;
+  a.req_idx = req_idx;
+  a.q = q;
+  a.k = k;
+  a.v = v;
+  a.io_bf16 = io_dtype == DASC_IO_BF16;
+  a.g = g;
+  a.beta = beta;
+  a.cu_seqlens = cu_seqlens;
+  a.n_req = n_req;
+  a.total_tokens = total_tokens;
+  a.max_seqlen = max_seqlen;
+  a.layer_begin = layer_begin;
+  a.n_layers_in_call = layer_end - layer_begin;
+  a.q_scale = q_scale;
+  a.o = o;
+  a.o_bf16 = o_dtype == DASC_IO_BF16;
+  a.mode = mode;
+  a.row_keep = plan->d_row_keep;
+  a.rows_per_layer = plan->rows_per_layer;
+  a.workspace = workspace;
+  a.workspace_bytes = workspace_bytes;
+
+  int e;
+  if (chunked) {
+    const size_t need = dasc_refresh_chunked_workspace_bytes(n_req, a.n_layers_in_call, a.H_v);
+    if (need && (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u)))
+      return DASC_ERR_WORKSPACE;
+    e = dasc_launch_refresh_chunked(a, cuda_stream);
+    if (e == -1) {
+      if (algo == DASC_ALGO_CHUNKED) return DASC_ERR_UNSUPPORTED;
+      e = dasc_launch_refresh_seq(a, cuda_stream);
+    }
+  } else {
+    e = dasc_launch_refresh_seq(a, cuda_stream);
+  }
+  if (e == -1) return DASC_ERR_SHAPE;
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+dasc_status_t dasc_refresh_status(const void *workspace, size_t workspace_bytes) {
+  if (!workspace || workspace_bytes < 4) return DASC_OK;  // nothing was recorded
+  uint32_t flag = 0;
+  if (cudaMemcpy(&flag, workspace, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return DASC_ERR_CUDA;
+  return flag == 0 ? DASC_OK : DASC_ERR_TIMEOUT;
+}
+
+const char *dasc_status_string(dasc_status_t s) {
+  switch (s) {
+    case DASC_OK: return "ok";
+    case DASC_ERR_INVALID_ARG: return "invalid argument";
+    case DASC_ERR_SHAPE: return "unsupported shape";
+    case DASC_ERR_UNSUPPORTED: return "not implemented";
+    case DASC_ERR_ALLOC: return "allocation failed";
+    case DASC_ERR_CUDA: return "CUDA error";
+    case DASC_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case DASC_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+const char *dasc_version(void) { return "0.1.0"; }
+
+}  // extern "C"

@@ -1,0 +1,128 @@
+// Store / Load copy kernels: pack (gather retained rows into the ragged pool) and
+// restore (scatter back with the zero-fill fused, every dense byte written once).
+// Both are pure HBM-bandwidth work: 128-bit streaming loads and stores, several
+// independent loads in flight per thread, index tables small enough to live in L2.
+#include <cuda_runtime.h>
+
+#include "dasc_internal.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) {
+  asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+               "r"(v.w)
+               : "memory");
+}
+
+// grid = (ceil(packed_vecs / (kThreads*UNROLL)), pairs).  A "vec" is 16 bytes of a row.
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads) pack_kernel(const uint4 *__restrict__ state, int64_t layer_stride4,
+                                                        int64_t req_stride4, const int32_t *__restrict__ src_req,
+                                                        uint4 *__restrict__ pool, int64_t slot_stride4,
+                                                        const int32_t *__restrict__ dst_slot,
+                                                        const DascRowSrc *__restrict__ row_src, uint32_t packed_vecs,
+                                                        uint32_t vecs_per_row, int32_t n_pairs) {
+  const uint32_t base = blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
+  for (int32_t pair = blockIdx.y; pair < n_pairs; pair += gridDim.y) {
+    const uint4 *src_base = state + static_cast<int64_t>(__ldg(src_req + pair)) * req_stride4;
+    uint4 *dst_base = pool + static_cast<int64_t>(__ldg(dst_slot + pair)) * slot_stride4;
+    uint4 val[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const uint32_t i = base + u * kThreads;
+      if (i < packed_vecs) {
+        const uint32_t row = i / vecs_per_row;
+        const uint32_t vec = i - row * vecs_per_row;
+        const int2 s = __ldg(reinterpret_cast<const int2 *>(row_src) + row);  // {layer, dense row}
+        val[u] = ld_stream(src_base + s.x * layer_stride4 + static_cast<int64_t>(s.y) * vecs_per_row + vec);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const uint32_t i = base + u * kThreads;
+      if (i < packed_vecs) st_stream(dst_base + i, val[u]);
+    }
+  }
+}
+
+// grid = (ceil(layer_vecs / (kThreads*UNROLL)), n_layers, pairs).
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads) restore_kernel(const uint4 *__restrict__ pool, int64_t slot_stride4,
+                                                           const int32_t *__restrict__ src_slot,
+                                                           uint4 *__restrict__ state, int64_t layer_stride4,
+                                                           int64_t req_stride4, const int32_t *__restrict__ dst_req,
+                                                           const int32_t *__restrict__ row_pos, uint32_t layer_vecs,
+                                                           uint32_t rows_per_layer, uint32_t vecs_per_row,
+                                                           int32_t n_pairs) {
+  const uint32_t base = blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
+  const int32_t layer = blockIdx.y;
+  const int32_t *pos_l = row_pos + static_cast<int64_t>(layer) * rows_per_layer;
+  for (int32_t pair = blockIdx.z; pair < n_pairs; pair += gridDim.z) {
+    const uint4 *src_base = pool + static_cast<int64_t>(__ldg(src_slot + pair)) * slot_stride4;
+    uint4 *dst_base = state + static_cast<int64_t>(__ldg(dst_req + pair)) * req_stride4 + layer * layer_stride4;
+    uint4 val[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const uint32_t i = base + u * kThreads;
+      val[u] = make_uint4(0u, 0u, 0u, 0u);  // omitted rows: +0.0f
+      if (i < layer_vecs) {
+        const uint32_t row = i / vecs_per_row;
+        const uint32_t vec = i - row * vecs_per_row;
+        const int32_t pos = __ldg(pos_l + row);
+        if (pos >= 0) val[u] = ld_stream(src_base + static_cast<int64_t>(pos) * vecs_per_row + vec);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const uint32_t i = base + u * kThreads;
+      if (i < layer_vecs) st_stream(dst_base + i, val[u]);
+    }
+  }
+}
+
+constexpr int kPackUnroll = 8;
+constexpr int kRestoreUnroll = 8;
+
+}  // namespace
+
+int dasc_launch_pack(const dasc_plan_s *plan, const float *state, int64_t layer_stride, int64_t req_stride,
+                     const int32_t *src_req, float *pool, int64_t slot_stride, const int32_t *dst_slot,
+                     int32_t n_pairs, void *stream) {
+  const uint32_t vpr = static_cast<uint32_t>(plan->info.d_v / 4);
+  const uint64_t packed_vecs = static_cast<uint64_t>(plan->packed_rows) * vpr;
+  if (packed_vecs == 0 || n_pairs == 0) return cudaSuccess;
+  const uint32_t per_block = kThreads * kPackUnroll;
+  dim3 grid(static_cast<uint32_t>((packed_vecs + per_block - 1) / per_block),
+            static_cast<uint32_t>(n_pairs < 65535 ? n_pairs : 65535));
+  pack_kernel<kPackUnroll><<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      reinterpret_cast<const uint4 *>(state), layer_stride / 4, req_stride / 4, src_req,
+      reinterpret_cast<uint4 *>(pool), slot_stride / 4, dst_slot, plan->d_row_src,
+      static_cast<uint32_t>(packed_vecs), vpr, n_pairs);
+  return static_cast<int>(cudaGetLastError());
+}
+
+int dasc_launch_restore(const dasc_plan_s *plan, const float *pool, int64_t slot_stride, const int32_t *src_slot,
+                        float *state, int64_t layer_stride, int64_t req_stride, const int32_t *dst_req,
+                        int32_t n_pairs, void *stream) {
+  const uint32_t vpr = static_cast<uint32_t>(plan->info.d_v / 4);
+  const uint64_t layer_vecs = static_cast<uint64_t>(plan->rows_per_layer) * vpr;
+  if (n_pairs == 0) return cudaSuccess;
+  const uint32_t per_block = kThreads * kRestoreUnroll;
+  dim3 grid(static_cast<uint32_t>((layer_vecs + per_block - 1) / per_block),
+            static_cast<uint32_t>(plan->info.n_layers), static_cast<uint32_t>(n_pairs < 65535 ? n_pairs : 65535));
+  restore_kernel<kRestoreUnroll><<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      reinterpret_cast<const uint4 *>(pool), slot_stride / 4, src_slot, reinterpret_cast<uint4 *>(state),
+      layer_stride / 4, req_stride / 4, dst_req, plan->d_row_pos, static_cast<uint32_t>(layer_vecs),
+      static_cast<uint32_t>(plan->rows_per_layer), vpr, n_pairs);
+  return static_cast<int>(cudaGetLastError());
+}
