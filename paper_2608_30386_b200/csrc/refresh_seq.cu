@@ -85,7 +85,9 @@ __global__ void __launch_bounds__(DV *RS) refresh_seq_kernel(DascRefreshArgs a) 
   const int layer = a.layer_begin + lc;
   const int64_t t_begin = a.cu_seqlens[r];
   const int n_tok = static_cast<int>(a.cu_seqlens[r + 1] - t_begin);
-  if (n_tok <= 0) return;  // an empty suffix leaves the state as it is in both modes
+  // An empty suffix continues nothing; in the scratch mode it still replaces the omitted
+  // units by the (all-zero) scratch state, as the definition says.
+  if (n_tok <= 0 && a.mode == DASC_REFRESH_CONTINUE) return;
 
   float *st = a.state + static_cast<int64_t>(a.req_idx[r]) * a.req_stride + static_cast<int64_t>(layer) * a.layer_stride +
               static_cast<int64_t>(h) * DK * DV;
@@ -137,8 +139,8 @@ __global__ void __launch_bounds__(DV *RS) refresh_seq_kernel(DascRefreshArgs a) 
     cp_async_commit();
   };
 
-  const int n_grp = (n_tok + TB - 1) / TB;
-  stage(0, 0);
+  const int n_grp = n_tok > 0 ? (n_tok + TB - 1) / TB : 0;
+  if (n_grp > 0) stage(0, 0);
   int parity = 0;  // token parity for the reduction buffers
   bool have_prev_o = false;
   int prev_t = 0;
