@@ -179,6 +179,7 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------------------
 
 def main():
+    global N_REQ, SUFFIX, KEEP, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
@@ -191,7 +192,6 @@ def main():
     ap.add_argument("--suffix", type=int, default=SUFFIX, help="profiling only: shrink the refresh suffix")
     ap.add_argument("--keep", type=float, default=KEEP, help="keep ratio (0.25, 0.38, 0.5, 1.0 in the sweep)")
     args = ap.parse_args()
-    global N_REQ, SUFFIX, KEEP, WORKLOAD
     if (args.requests, args.suffix, args.keep) != (N_REQ, SUFFIX, KEEP):
         N_REQ, SUFFIX, KEEP = args.requests, args.suffix, args.keep
         WORKLOAD = f"kda_24x32x128x128_fp32_{N_REQ}req_keep{KEEP}_suffix{SUFFIX}_bf16"
