@@ -10,7 +10,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdasc.so")
 SOURCES = ["dasc_api.cu", "plan_host.cpp", "pack_restore.cu", "refresh_seq.cu", "refresh_chunked.cu"]
-HEADERS = [os.path.join(ROOT, "include", "dasc.h"), os.path.join(CSRC, "dasc_internal.h")]
+HEADERS = [os.path.join(ROOT, "include", "dasc.h"), os.path.join(CSRC, "dasc_internal.h"),
+           os.path.join(CSRC, "tcgen05_util.cuh")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

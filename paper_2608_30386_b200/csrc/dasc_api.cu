@@ -189,8 +189,10 @@ dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t l
   const size_t esz = io_dtype == DASC_IO_BF16 ? 2 : 4;
   if ((plan->info.d_k * esz) % 16 || (plan->info.d_v * esz) % 16) return DASC_ERR_SHAPE;
 
-  bool chunked = algo == DASC_ALGO_CHUNKED || (algo == DASC_ALGO_AUTO && chunked_shape_ok(plan));
-  if (algo == DASC_ALGO_CHUNKED && !chunked_shape_ok(plan)) return DASC_ERR_SHAPE;
+  // the chunked kernel takes d_k = d_v = 128 and bf16 token streams
+  const bool chunked_ok = chunked_shape_ok(plan) && io_dtype == DASC_IO_BF16;
+  if (algo == DASC_ALGO_CHUNKED && !chunked_ok) return DASC_ERR_SHAPE;
+  const bool chunked = algo == DASC_ALGO_CHUNKED || (algo == DASC_ALGO_AUTO && chunked_ok);
 
   DascRefreshArgs a{};
   a.kind = plan->info.kind;
