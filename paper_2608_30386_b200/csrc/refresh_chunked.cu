@@ -10,18 +10,23 @@
 //   S_C  = Diag(exp(G_C - G_m)) (S' + Kh^T U)
 // Referencing the decay to the midpoint keeps every exponent within half a chunk's decay.
 //
-// Mapping.  One CTA (128 threads) per (request, layer, value head); the state lives in TMEM
-// transposed, S'^T: lane = value column v, column = key channel c, fp32, for the whole suffix.
-// All five products run as M = 128 tcgen05.mma (kind::tf32, fp32 accumulate) with the value
-// index on the TMEM lanes, so that each accumulator is directly the A operand of the next:
+// Mapping.  One CTA per (request, layer, value head): eight compute warps (256 threads) and
+// one warp that only issues tensor-core work.  The state lives in TMEM transposed, S'^T:
+// lane = value column v, column = key channel c, fp32, for the whole suffix.  All five
+// products run as M = 128 tcgen05.mma (kind::tf32, fp32 accumulate) with the value index on
+// the TMEM lanes, so that each accumulator is directly the A operand of the next:
 //   MMA1  [Kt;Qt] Kh^T            -> A (lanes 0-63) and P (lanes 64-127)        smem x smem
 //   MMA2  S'^T [Kt;Qt]^T          -> R^T | (Qt S')^T                            tmem x smem
 //   MMA3  RHS^T T^T               -> U^T                                         tmem x smem
 //   MMA4  (Qt S')^T += U^T P^T    -> O^T                                         tmem x smem
 //   MMA5  S'^T      += U^T Kh     -> state                                       tmem x smem
 // Operands built on the CUDA cores are rounded to tf32 (round-to-nearest) before use; the
-// state master copy stays fp32.  The unit-lower-triangular inverse T = (I + A)^-1 is computed
-// in fp32 on the CUDA cores (16x16 diagonal blocks by substitution, the rest blockwise).
+// state master copy stays fp32.  The unit-lower-triangular inverse T = (I + A)^-1 is formed
+// blockwise: 16x16 diagonal blocks by fp32 substitution, off-diagonal blocks by warp-level
+// mma.sync (tf32) products.  Token inputs of chunk n+1 are fetched with cp.async while chunk n
+// computes: q, k into their own buffer, g into the triangular work matrices once T is out,
+// v into the V tile once the right-hand side is formed.  Kh[t][c] (needed by MMA1 only)
+// shares its storage with the T and P tiles (written after MMA1 has completed).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -32,33 +37,55 @@ namespace {
 
 using namespace tc5;
 
-constexpr int C = 64;     // chunk length
-constexpr int D = 128;    // d_k = d_v
-constexpr int NT = 128;   // threads per CTA
-constexpr int LDX = 68;   // row pitch (floats) of the fp32 triangular work matrices
+constexpr int C = 64;        // chunk length
+constexpr int D = 128;       // d_k = d_v
+constexpr int NC = 256;      // compute threads
+constexpr int NT = NC + 32;  // + the MMA-issuing warp
+constexpr int LDX = 68;      // row pitch (floats) of the fp32 triangular work matrices
 
 // TMEM columns
 constexpr uint32_t COL_S = 0, COL_SOP = 128, COL_RO = 256, COL_AP = 384, COL_U = 448;
 
 // shared memory map (bytes)
-constexpr uint32_t OFF_KQ = 0;                       // [4][128 rows][128 B]  rows 0-63 Kt, 64-127 Qt
-constexpr uint32_t OFF_KH = OFF_KQ + 4 * 128 * 128;  // [4][64 rows][128 B]   Kh[t][c]
-constexpr uint32_t OFF_KHT = OFF_KH + 4 * 64 * 128;  // [2][128 rows][128 B]  Kh^T[c][t]
-constexpr uint32_t OFF_TM = OFF_KHT + 2 * 128 * 128; // [2][64 rows][128 B]   T[t][i]
-constexpr uint32_t OFF_PM = OFF_TM + 2 * 64 * 128;   // [2][64 rows][128 B]   P[t][i]
-constexpr uint32_t OFF_V = OFF_PM + 2 * 64 * 128;    // [64][128] bf16
-constexpr uint32_t OFF_L = OFF_V + C * D * 2;        // [64][LDX] fp32
-constexpr uint32_t OFF_X = OFF_L + C * LDX * 4;      // [64][LDX] fp32
-constexpr uint32_t OFF_FAC = OFF_X + C * LDX * 4;    // [128] fp32 state factor per channel
-constexpr uint32_t OFF_BETA = OFF_FAC + D * 4;       // [64] fp32
-constexpr uint32_t OFF_MISC = OFF_BETA + C * 4;      // barriers, tmem base, abort flag
-constexpr uint32_t SMEM_BYTES = OFF_MISC + 64;
-constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;   // slack to align the base to 1024 bytes
+constexpr uint32_t OFF_KQ = 0;                        // [4][128 rows][128 B]  rows 0-63 Kt, 64-127 Qt; later the O tile
+constexpr uint32_t OFF_KHT = OFF_KQ + 4 * 128 * 128;  // [2][128 rows][128 B]  Kh^T[c][t]
+constexpr uint32_t OFF_KH = OFF_KHT + 2 * 128 * 128;  // [4][64 rows][128 B]   Kh[t][c], until MMA1 is done; then:
+constexpr uint32_t OFF_TM = OFF_KH;                   // [2][64 rows][128 B]   T[t][i]
+constexpr uint32_t OFF_PM = OFF_TM + 2 * 64 * 128;    // [2][64 rows][128 B]   P[t][i]
+constexpr uint32_t OFF_RAWQ = OFF_KH + 4 * 64 * 128;  // [64][128] bf16 raw q of the next chunk
+constexpr uint32_t OFF_RAWK = OFF_RAWQ + C * D * 2;   // [64][128] bf16 raw k of the next chunk
+constexpr uint32_t OFF_V = OFF_RAWK + C * D * 2;      // [64][128] bf16
+constexpr uint32_t OFF_L = OFF_V + C * D * 2;         // [64][LDX] fp32                  (raw g of the next chunk
+constexpr uint32_t OFF_X = OFF_L + C * LDX * 4;       // [64][LDX] fp32                   spans L and X)
+constexpr uint32_t OFF_FAC = OFF_X + C * LDX * 4;     // [128] fp32 state factor per channel
+constexpr uint32_t OFF_POST = OFF_FAC + D * 4;        // [2][128] fp32 log-factor owed after a chunk, by chunk parity
+constexpr uint32_t OFF_BETA = OFF_POST + 2 * D * 4;   // [2][64] fp32, by chunk parity
+constexpr uint32_t OFF_GSC = OFF_BETA + 2 * C * 4;    // [2][64] fp32 scalar log-decay (GDN), by chunk parity
+constexpr uint32_t OFF_MISC = OFF_GSC + 2 * C * 4;    // barriers, tmem base, abort flag
+constexpr uint32_t SMEM_BYTES = OFF_MISC + 128;
+constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;    // slack to align the base to 1024 bytes
+static_assert(2 * C * LDX * 4 >= C * D * 4, "raw g must fit in the L and X matrices");
+static_assert(SMEM_ALLOC <= 227 * 1024, "shared memory budget");
 
 constexpr uint32_t kMaxPolls = 1u << 22;
 
+// Optional per-phase cycle counters of CTA 0 (development builds only): accumulated by thread 0
+// and written behind the time-out flag in the workspace.
+#ifdef DASC_PHASE_TIMING
+#define PT_DECL long long pt_acc[16] = {0}; long long pt_last = clock64();
+#define PT(i) do { long long pt_now = clock64(); pt_acc[i] += pt_now - pt_last; pt_last = pt_now; } while (0)
+#define PT_DUMP do { if (blockIdx.x == 0 && tid == 0) { long long *d = reinterpret_cast<long long *>(static_cast<char *>(a.workspace) + 64); for (int i = 0; i < 16; ++i) d[i] = pt_acc[i]; } } while (0)
+#else
+#define PT_DECL
+#define PT(i)
+#define PT_DUMP
+#endif
+
 struct Misc {
+  // tensor core -> compute warps (one tcgen05.commit each per chunk)
   uint64_t bar_ap, bar_ro, bar_u, bar_os;
+  // compute warps -> issuing warp (256 arrivals each per chunk)
+  uint64_t rdy_prep, rdy_state, rdy_rhs, rdy_u;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -74,7 +101,14 @@ __device__ __forceinline__ void cp_async16_zfill(uint32_t smem, const void *gmem
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem), "l"(gmem), "r"(n) : "memory");
 }
 
-// Bounded wait on an MMA-completion barrier; after one time-out every later wait returns at once.
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// barrier among the 256 compute threads only
+__device__ __forceinline__ void sync_compute() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// Bounded wait; after one time-out every later wait of this CTA returns at once.
 __device__ __forceinline__ void wait_bar(uint64_t *bar, uint32_t parity, Misc *misc, uint32_t *err) {
   if (misc->abort_flag) return;
   if (!mbar_wait_bounded(bar, parity, kMaxPolls)) {
@@ -83,25 +117,38 @@ __device__ __forceinline__ void wait_bar(uint64_t *bar, uint32_t parity, Misc *m
   }
 }
 
-// C (16x16, at c) = sign * sum_p A_p B_p over `np` block pairs; 64 threads, thread (i, jq) -> C[i][4jq..4jq+3].
-__device__ __forceinline__ void block_mm(float *c, const float *const *a, const float *const *b, int np, float sign,
-                                         int id) {
-  const int i = id >> 2, j0 = (id & 3) << 2;
-  float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-  for (int p = 0; p < np; ++p) {
-    const float *ap = a[p] + i * LDX;
-    const float *bp = b[p] + j0;
+__device__ __forceinline__ void mma_tf32_16x8x8(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// One warp: acc (16x16) += A (16x16) * B (16x16), blocks in shared memory with pitch LDX.
+__device__ __forceinline__ void warp_mm_acc(float (&acc)[2][4], const float *A, const float *B, int lane) {
+  const int g = lane >> 2, tig = lane & 3;
 #pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      const float av = ap[k];
-      const float4 bv = *reinterpret_cast<const float4 *>(bp + k * LDX);
-      acc0 = fmaf(av, bv.x, acc0);
-      acc1 = fmaf(av, bv.y, acc1);
-      acc2 = fmaf(av, bv.z, acc2);
-      acc3 = fmaf(av, bv.w, acc3);
+  for (int kh = 0; kh < 2; ++kh) {
+    uint32_t af[4];
+    af[0] = to_tf32(A[g * LDX + 8 * kh + tig]);
+    af[1] = to_tf32(A[(g + 8) * LDX + 8 * kh + tig]);
+    af[2] = to_tf32(A[g * LDX + 8 * kh + tig + 4]);
+    af[3] = to_tf32(A[(g + 8) * LDX + 8 * kh + tig + 4]);
+#pragma unroll
+    for (int nh = 0; nh < 2; ++nh) {
+      uint32_t bf[2];
+      bf[0] = to_tf32(B[(8 * kh + tig) * LDX + 8 * nh + g]);
+      bf[1] = to_tf32(B[(8 * kh + tig + 4) * LDX + 8 * nh + g]);
+      mma_tf32_16x8x8(acc[nh], af, bf);
     }
   }
-  *reinterpret_cast<float4 *>(c + i * LDX + j0) = make_float4(sign * acc0, sign * acc1, sign * acc2, sign * acc3);
+}
+__device__ __forceinline__ void warp_mm_store(float *Cb, const float (&acc)[2][4], float sign, int lane) {
+  const int g = lane >> 2, tig = lane & 3;
+#pragma unroll
+  for (int nh = 0; nh < 2; ++nh) {
+    *reinterpret_cast<float2 *>(Cb + g * LDX + 8 * nh + 2 * tig) = make_float2(sign * acc[nh][0], sign * acc[nh][1]);
+    *reinterpret_cast<float2 *>(Cb + (g + 8) * LDX + 8 * nh + 2 * tig) = make_float2(sign * acc[nh][2], sign * acc[nh][3]);
+  }
 }
 
 template <bool KDA, typename OT>
@@ -112,12 +159,17 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
   float *Lm = reinterpret_cast<float *>(smem + OFF_L);
   float *Xm = reinterpret_cast<float *>(smem + OFF_X);
   float *fac_s = reinterpret_cast<float *>(smem + OFF_FAC);
+  float *post_s = reinterpret_cast<float *>(smem + OFF_POST);
   float *beta_s = reinterpret_cast<float *>(smem + OFF_BETA);
+  float *gsc_s = reinterpret_cast<float *>(smem + OFF_GSC);
   const __nv_bfloat16 *Vs = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_V);
+  const __nv_bfloat16 *Qraw = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_RAWQ);
+  const __nv_bfloat16 *Kraw = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_RAWK);
+  const float *Graw = reinterpret_cast<const float *>(smem + OFF_L);
   Misc *misc = reinterpret_cast<Misc *>(smem + OFF_MISC);
   uint32_t *err = static_cast<uint32_t *>(a.workspace);
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.x % a.H_v;
   const int lc = (blockIdx.x / a.H_v) % a.n_layers_in_call;
   const int r = blockIdx.x / (a.H_v * a.n_layers_in_call);
@@ -145,10 +197,14 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
     mbar_init(&misc->bar_ro, 1);
     mbar_init(&misc->bar_u, 1);
     mbar_init(&misc->bar_os, 1);
+    mbar_init(&misc->rdy_prep, NC);
+    mbar_init(&misc->rdy_state, NC);
+    mbar_init(&misc->rdy_rhs, NC);
+    mbar_init(&misc->rdy_u, NC);
     misc->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 0) {
+  if (warp == 8) {
     tmem_alloc(&misc->tmem_base, 512);
     tmem_relinquish();
   }
@@ -156,364 +212,470 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tm = misc->tmem_base;
-  const uint32_t tlane = tm + (static_cast<uint32_t>(warp * 32) << 16);  // this warp's lane quadrant
+  const int n_chunks = (n_tok + C - 1) / C;
 
   constexpr uint32_t ID_M128_N64 = idesc_tf32(128, 64, false, false);
   constexpr uint32_t ID_M128_N128 = idesc_tf32(128, 128, false, false);
-  constexpr float LOG2E = 1.4426950408889634f;
 
-  float prev_post = 0.f;  // thread c: log of the factor still owed to channel c of the state
-  const int n_chunks = (n_tok + C - 1) / C;
-
-  for (int ch = 0; ch < n_chunks; ++ch) {
-    const uint32_t par = ch & 1;
-    const int t0 = ch * C;
-    const int ntok = min(C, n_tok - t0);
-
-    // ---- (1) V tile and beta for this chunk (used in step 7) ----
-    for (int i = tid; i < C * (D * 2 / 16); i += NT) {
-      const int t = i >> 4, j = i & 15;
-      const bool valid = t < ntok;
-      cp_async16_zfill(sbase + OFF_V + t * (D * 2) + j * 16,
-                       reinterpret_cast<const char *>(gv + (t0 + (valid ? t : 0)) * v_stride) + j * 16, valid);
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    if (tid < C) beta_s[tid] = tid < ntok ? gb[(t0 + tid) * b_stride] : 0.f;
-
-    // ---- (2) prep: thread = key channel c ----
-    {
-      const int c = tid;
-      float G[C];
+  if (warp == 8) {
+    // =========================== tensor-core issue warp ===========================
+    for (int ch = 0; ch < n_chunks; ++ch) {
+      const uint32_t par = ch & 1;
+      // MMA1: [Kt;Qt] Kh^T
+      if (lane == 0) wait_bar(&misc->rdy_prep, par, misc, err);
+      __syncwarp();
+      if (lane == 0) {
+        tc_fence_after_sync();
 #pragma unroll
-      for (int t = 0; t < C; ++t) G[t] = t < ntok ? gg[(t0 + t) * g_stride + (KDA ? c : 0)] : 0.f;
+        for (int kb = 0; kb < 4; ++kb)
 #pragma unroll
-      for (int t = 1; t < C; ++t) G[t] += G[t - 1];
-      const float Gm = G[C / 2 - 1], Gc = G[C - 1];
-      fac_s[c] = ex2f((prev_post + Gm) * LOG2E);
-      prev_post = Gc - Gm;
-#pragma unroll
-      for (int t4 = 0; t4 < C; t4 += 4) {
-        uint32_t kht[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int t = t4 + u;
-          float kf = 0.f, qf = 0.f;
-          if (t < ntok) {
-            kf = __bfloat162float(gk[(t0 + t) * qk_stride + c]);
-            qf = __bfloat162float(gq[(t0 + t) * qk_stride + c]) * a.q_scale;
-          }
-          const float d = (G[t] - Gm) * LOG2E;
-          const float e1 = ex2f(d), e2 = ex2f(-d);
-          *reinterpret_cast<uint32_t *>(smem + OFF_KQ + sw128_offset(128, t, c)) = to_tf32(kf * e1);
-          *reinterpret_cast<uint32_t *>(smem + OFF_KQ + sw128_offset(128, 64 + t, c)) = to_tf32(qf * e1);
-          kht[u] = to_tf32(kf * e2);
-          *reinterpret_cast<uint32_t *>(smem + OFF_KH + sw128_offset(64, t, c)) = kht[u];
-        }
-        *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c, t4)) = make_uint4(kht[0], kht[1], kht[2], kht[3]);
+          for (int j = 0; j < 4; ++j)
+            mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + kb * (128 * 128) + j * 32),
+                   desc_kmajor(sbase + OFF_KH + kb * (64 * 128) + j * 32), ID_M128_N64, (kb | j) != 0);
+        mma_commit(&misc->bar_ap);
       }
-    }
-    fence_smem_to_async();
-    __syncthreads();
-
-    // ---- (3) MMA1: [Kt;Qt] Kh^T ----
-    if (tid == 0) {
-      tc_fence_after_sync();
+      // MMA2: S'^T [Kt;Qt]^T
+      if (lane == 0) wait_bar(&misc->rdy_state, par, misc, err);
+      __syncwarp();
+      if (lane == 0) {
+        tc_fence_after_sync();
 #pragma unroll
-      for (int kb = 0; kb < 4; ++kb)
+        for (int kb = 0; kb < 4; ++kb)
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + kb * (128 * 128) + j * 32),
-                 desc_kmajor(sbase + OFF_KH + kb * (64 * 128) + j * 32), ID_M128_N64, (kb | j) != 0);
-      mma_commit(&misc->bar_ap);
-    }
-
-    // ---- (4) state pass: thread = value column v; scale to this chunk's midpoint, refresh the tf32 copy ----
-    {
-      const int v = tid;
-#pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
-        uint32_t s[32];
-        if (ch == 0) {
-          if (a.mode == DASC_REFRESH_CONTINUE) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) s[j] = __float_as_uint(st[(c0 + j) * D + v]);
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) s[j] = 0u;
-          }
-        } else {
-          tmem_ld32(tlane + COL_S + c0, s);
-          tmem_ld_wait();
-        }
-        uint32_t sop[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float x = __uint_as_float(s[j]) * fac_s[c0 + j];
-          s[j] = __float_as_uint(x);
-          sop[j] = to_tf32(x);
-        }
-        tmem_st32(tlane + COL_S + c0, s);
-        tmem_st32(tlane + COL_SOP + c0, sop);
+          for (int j = 0; j < 4; ++j)
+            mma_ts(tm + COL_RO, tm + COL_SOP + kb * 32 + j * 8, desc_kmajor(sbase + OFF_KQ + kb * (128 * 128) + j * 32),
+                   ID_M128_N128, (kb | j) != 0);
+        mma_commit(&misc->bar_ro);
       }
-      tmem_st_wait();
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-
-    // ---- (5) MMA2: S'^T [Kt;Qt]^T ----
-    if (tid == 0) {
-      tc_fence_after_sync();
-#pragma unroll
-      for (int kb = 0; kb < 4; ++kb)
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          mma_ts(tm + COL_RO, tm + COL_SOP + kb * 32 + j * 8, desc_kmajor(sbase + OFF_KQ + kb * (128 * 128) + j * 32),
-                 ID_M128_N128, (kb | j) != 0);
-      mma_commit(&misc->bar_ro);
-    }
-
-    // ---- (6) A and P out of TMEM; T = (I + A)^-1 ----
-    wait_bar(&misc->bar_ap, par, misc, err);
-    tc_fence_after_sync();
-    if (tid < C) {
-      // lanes 0-63: row t of A = strict_lower(Kt Kh^T) * beta_t, kept in fp32 for the inverse
-      const int t = tid;
-      const float bt = beta_s[t];
-#pragma unroll 1
-      for (int c0 = 0; c0 < C; c0 += 32) {
-        uint32_t x[32];
-        tmem_ld32(tlane + COL_AP + c0, x);
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          float4 o;
-          o.x = (c0 + j + 0 < t) ? bt * __uint_as_float(x[j + 0]) : 0.f;
-          o.y = (c0 + j + 1 < t) ? bt * __uint_as_float(x[j + 1]) : 0.f;
-          o.z = (c0 + j + 2 < t) ? bt * __uint_as_float(x[j + 2]) : 0.f;
-          o.w = (c0 + j + 3 < t) ? bt * __uint_as_float(x[j + 3]) : 0.f;
-          *reinterpret_cast<float4 *>(Lm + t * LDX + c0 + j) = o;
-        }
-      }
-    } else {
-      // lanes 64-127: row t of P = lower_incl_diag(Qt Kh^T), straight to its operand tile
-      const int t = tid - C;
-#pragma unroll 1
-      for (int c0 = 0; c0 < C; c0 += 32) {
-        uint32_t x[32];
-        tmem_ld32(tlane + COL_AP + c0, x);
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          uint4 o;
-          o.x = (c0 + j + 0 <= t) ? to_tf32(__uint_as_float(x[j + 0])) : 0u;
-          o.y = (c0 + j + 1 <= t) ? to_tf32(__uint_as_float(x[j + 1])) : 0u;
-          o.z = (c0 + j + 2 <= t) ? to_tf32(__uint_as_float(x[j + 2])) : 0u;
-          o.w = (c0 + j + 3 <= t) ? to_tf32(__uint_as_float(x[j + 3])) : 0u;
-          *reinterpret_cast<uint4 *>(smem + OFF_PM + sw128_offset(64, t, c0 + j)) = o;
-        }
-      }
-    }
-    __syncthreads();
-    // diagonal 16x16 blocks: thread (block b, column cc) solves (I + L_bb) x = e_cc by forward substitution
-    if (tid < C) {
-      const int b = tid >> 4, cc = tid & 15;
-      const float *Lb = Lm + (b * 16) * LDX + b * 16;
-      float x[16];
-#pragma unroll
-      for (int rr = 0; rr < 16; ++rr) {
-        float acc = (rr == cc) ? 1.f : 0.f;
-#pragma unroll
-        for (int j = 0; j < rr; ++j) acc = fmaf(-Lb[rr * LDX + j], x[j], acc);
-        x[rr] = acc;
-      }
-#pragma unroll
-      for (int rr = 0; rr < 16; ++rr) Xm[(b * 16 + rr) * LDX + b * 16 + cc] = x[rr];
-    }
-    __syncthreads();
-    {
-      // off-diagonal blocks; Y_IJ = sum_K L_IK X_KJ is parked in the (unused) upper block (J, I) of X
-      const int grp = tid >> 6, id = tid & 63;
-      auto Lb = [&](int I, int J) { return Lm + (I * 16) * LDX + J * 16; };
-      auto Xb = [&](int I, int J) { return Xm + (I * 16) * LDX + J * 16; };
-      const float *pa[3];
-      const float *pb[3];
-      // first sub-diagonal
-      if (grp == 0) {
-        pa[0] = Lb(1, 0); pb[0] = Xb(0, 0); block_mm(Xb(0, 1), pa, pb, 1, 1.f, id);
-        pa[0] = Lb(3, 2); pb[0] = Xb(2, 2); block_mm(Xb(2, 3), pa, pb, 1, 1.f, id);
-      } else {
-        pa[0] = Lb(2, 1); pb[0] = Xb(1, 1); block_mm(Xb(1, 2), pa, pb, 1, 1.f, id);
-      }
-      __syncthreads();
-      if (grp == 0) {
-        pa[0] = Xb(1, 1); pb[0] = Xb(0, 1); block_mm(Xb(1, 0), pa, pb, 1, -1.f, id);
-        pa[0] = Xb(3, 3); pb[0] = Xb(2, 3); block_mm(Xb(3, 2), pa, pb, 1, -1.f, id);
-      } else {
-        pa[0] = Xb(2, 2); pb[0] = Xb(1, 2); block_mm(Xb(2, 1), pa, pb, 1, -1.f, id);
-      }
-      __syncthreads();
-      // second sub-diagonal
-      if (grp == 0) {
-        pa[0] = Lb(2, 0); pb[0] = Xb(0, 0); pa[1] = Lb(2, 1); pb[1] = Xb(1, 0); block_mm(Xb(0, 2), pa, pb, 2, 1.f, id);
-      } else {
-        pa[0] = Lb(3, 1); pb[0] = Xb(1, 1); pa[1] = Lb(3, 2); pb[1] = Xb(2, 1); block_mm(Xb(1, 3), pa, pb, 2, 1.f, id);
-      }
-      __syncthreads();
-      if (grp == 0) {
-        pa[0] = Xb(2, 2); pb[0] = Xb(0, 2); block_mm(Xb(2, 0), pa, pb, 1, -1.f, id);
-      } else {
-        pa[0] = Xb(3, 3); pb[0] = Xb(1, 3); block_mm(Xb(3, 1), pa, pb, 1, -1.f, id);
-      }
-      __syncthreads();
-      // corner block
-      if (grp == 0) {
-        pa[0] = Lb(3, 0); pb[0] = Xb(0, 0); pa[1] = Lb(3, 1); pb[1] = Xb(1, 0); pa[2] = Lb(3, 2); pb[2] = Xb(2, 0);
-        block_mm(Xb(0, 3), pa, pb, 3, 1.f, id);
-      }
-      __syncthreads();
-      if (grp == 0) {
-        pa[0] = Xb(3, 3); pb[0] = Xb(0, 3); block_mm(Xb(3, 0), pa, pb, 1, -1.f, id);
-      }
-      __syncthreads();
-      // T (lower triangle of X, unit diagonal) -> tf32 operand tile
-      const int t = tid >> 1, i0 = (tid & 1) * 32;
-#pragma unroll
-      for (int j = 0; j < 32; j += 4) {
-        const float4 xv = *reinterpret_cast<const float4 *>(Xm + t * LDX + i0 + j);
-        uint4 o;
-        o.x = (i0 + j + 0 <= t) ? to_tf32(xv.x) : 0u;
-        o.y = (i0 + j + 1 <= t) ? to_tf32(xv.y) : 0u;
-        o.z = (i0 + j + 2 <= t) ? to_tf32(xv.z) : 0u;
-        o.w = (i0 + j + 3 <= t) ? to_tf32(xv.w) : 0u;
-        *reinterpret_cast<uint4 *>(smem + OFF_TM + sw128_offset(64, t, i0 + j)) = o;
-      }
-    }
-    fence_smem_to_async();
-
-    // ---- (7) RHS^T = beta (V - R)^T, written over R^T as the tf32 A operand of MMA3 ----
-    wait_bar(&misc->bar_ro, par, misc, err);
-    tc_fence_after_sync();
-    asm volatile("cp.async.wait_all;" ::: "memory");
-    __syncthreads();  // V tile visible to everyone
-    {
-      const int v = tid;
-#pragma unroll 1
-      for (int c0 = 0; c0 < C; c0 += 32) {
-        uint32_t x[32];
-        tmem_ld32(tlane + COL_RO + c0, x);
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float vv = __bfloat162float(Vs[(c0 + j) * D + v]);
-          x[j] = to_tf32(beta_s[c0 + j] * (vv - __uint_as_float(x[j])));
-        }
-        tmem_st32(tlane + COL_RO + c0, x);
-      }
-      tmem_st_wait();
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-
-    // ---- (8) MMA3: U^T = RHS^T T^T ----
-    if (tid == 0) {
-      tc_fence_after_sync();
-#pragma unroll
-      for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          mma_ts(tm + COL_U, tm + COL_RO + kb * 32 + j * 8, desc_kmajor(sbase + OFF_TM + kb * (64 * 128) + j * 32),
-                 ID_M128_N64, (kb | j) != 0);
-      mma_commit(&misc->bar_u);
-    }
-
-    // ---- (9) U^T rounded to tf32 in place ----
-    wait_bar(&misc->bar_u, par, misc, err);
-    tc_fence_after_sync();
-#pragma unroll 1
-    for (int c0 = 0; c0 < C; c0 += 32) {
-      uint32_t x[32];
-      tmem_ld32(tlane + COL_U + c0, x);
-      tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 32; ++j) x[j] = to_tf32(__uint_as_float(x[j]));
-      tmem_st32(tlane + COL_U + c0, x);
-    }
-    tmem_st_wait();
-    tc_fence_before_sync();
-    __syncthreads();
-
-    // ---- (10) MMA4: O^T += U^T P^T;  MMA5: S'^T += U^T Kh ----
-    if (tid == 0) {
-      tc_fence_after_sync();
-      if (go) {
+      // MMA3: U^T = RHS^T T^T
+      if (lane == 0) wait_bar(&misc->rdy_rhs, par, misc, err);
+      __syncwarp();
+      if (lane == 0) {
+        tc_fence_after_sync();
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
           for (int j = 0; j < 4; ++j)
-            mma_ts(tm + COL_RO + 64, tm + COL_U + kb * 32 + j * 8, desc_kmajor(sbase + OFF_PM + kb * (64 * 128) + j * 32),
-                   ID_M128_N64, true);
+            mma_ts(tm + COL_U, tm + COL_RO + kb * 32 + j * 8, desc_kmajor(sbase + OFF_TM + kb * (64 * 128) + j * 32),
+                   ID_M128_N64, (kb | j) != 0);
+        mma_commit(&misc->bar_u);
       }
+      // MMA4: O^T += U^T P^T;  MMA5: S'^T += U^T Kh
+      if (lane == 0) wait_bar(&misc->rdy_u, par, misc, err);
+      __syncwarp();
+      if (lane == 0) {
+        tc_fence_after_sync();
+        if (go) {
 #pragma unroll
-      for (int kb = 0; kb < 2; ++kb)
+          for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          mma_ts(tm + COL_S, tm + COL_U + kb * 32 + j * 8, desc_kmajor(sbase + OFF_KHT + kb * (128 * 128) + j * 32),
-                 ID_M128_N128, true);
-      mma_commit(&misc->bar_os);
+            for (int j = 0; j < 4; ++j)
+              mma_ts(tm + COL_RO + 64, tm + COL_U + kb * 32 + j * 8,
+                     desc_kmajor(sbase + OFF_PM + kb * (64 * 128) + j * 32), ID_M128_N64, true);
+        }
+#pragma unroll
+        for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            mma_ts(tm + COL_S, tm + COL_U + kb * 32 + j * 8, desc_kmajor(sbase + OFF_KHT + kb * (128 * 128) + j * 32),
+                   ID_M128_N128, true);
+        mma_commit(&misc->bar_os);
+      }
+      __syncwarp();
     }
+  } else {
+    // =============================== compute warps ===============================
+    const int quad = warp & 3, colh = warp >> 2;                           // TMEM lane quadrant, column half
+    const uint32_t tlane = tm + (static_cast<uint32_t>(quad * 32) << 16);  // this warp's TMEM lanes
+    const int vrow = quad * 32 + lane;                                     // the TMEM lane this thread owns
+    constexpr float LOG2E = 1.4426950408889634f;
+    PT_DECL
 
-    // ---- (11) outputs of this chunk ----
-    wait_bar(&misc->bar_os, par, misc, err);
-    tc_fence_after_sync();
-    if (go) {
-      const int v = tid;
-#pragma unroll 1
-      for (int c0 = 0; c0 < C; c0 += 32) {
-        uint32_t x[32];
-        tmem_ld32(tlane + COL_RO + 64 + c0, x);
-        tmem_ld_wait();
+    // cp.async stages of one chunk's inputs
+    auto stage_qk = [&](int ch) {
+      const int t0 = ch * C, ntok = min(C, n_tok - t0);
+      for (int i = tid; i < C * 16; i += NC) {
+        const int t = i >> 4, j = i & 15;
+        const bool valid = t < ntok;
+        const int64_t tt = t0 + (valid ? t : 0);
+        cp_async16_zfill(sbase + OFF_RAWQ + t * 256 + j * 16, reinterpret_cast<const char *>(gq + tt * qk_stride) + j * 16, valid);
+        cp_async16_zfill(sbase + OFF_RAWK + t * 256 + j * 16, reinterpret_cast<const char *>(gk + tt * qk_stride) + j * 16, valid);
+      }
+    };
+    auto stage_g = [&](int ch) {
+      const int t0 = ch * C, ntok = min(C, n_tok - t0);
+      if constexpr (KDA) {
+        for (int i = tid; i < C * 32; i += NC) {
+          const int t = i >> 5, j = i & 31;
+          const bool valid = t < ntok;
+          cp_async16_zfill(sbase + OFF_L + t * 512 + j * 16,
+                           reinterpret_cast<const char *>(gg + (t0 + (valid ? t : 0)) * g_stride) + j * 16, valid);
+        }
+      }
+    };
+    auto stage_v = [&](int ch) {
+      const int t0 = ch * C, ntok = min(C, n_tok - t0);
+      for (int i = tid; i < C * 16; i += NC) {
+        const int t = i >> 4, j = i & 15;
+        const bool valid = t < ntok;
+        cp_async16_zfill(sbase + OFF_V + t * 256 + j * 16,
+                         reinterpret_cast<const char *>(gv + (t0 + (valid ? t : 0)) * v_stride) + j * 16, valid);
+      }
+    };
+    // per-token scalars of a chunk (beta, and the scalar log-decay of GDN): threads 0-63 / 64-127
+    auto load_scalar = [&](int ch) -> float {
+      const int t0 = ch * C, ntok = min(C, n_tok - t0);
+      if (tid < C) return tid < ntok ? gb[(t0 + tid) * b_stride] : 0.f;
+      if (!KDA && tid < 2 * C) return (tid - C) < ntok ? gg[(t0 + tid - C) * g_stride] : 0.f;
+      return 0.f;
+    };
+    auto store_scalar = [&](int ch, float x) {
+      if (tid < C) beta_s[(ch & 1) * C + tid] = x;
+      else if (!KDA && tid < 2 * C) gsc_s[(ch & 1) * C + tid - C] = x;
+    };
+
+    if (n_chunks > 0) {
+      stage_qk(0);
+      stage_g(0);
+      stage_v(0);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      store_scalar(0, load_scalar(0));
+    }
+    if (tid < D) post_s[tid] = 0.f;  // nothing owed before the first chunk (parity 1 = "chunk -1")
+    if (tid < D) post_s[D + tid] = 0.f;
+
+    for (int ch = 0; ch < n_chunks; ++ch) {
+      const uint32_t par = ch & 1;
+      const int t0 = ch * C;
+      const int ntok = min(C, n_tok - t0);
+      const bool more = ch + 1 < n_chunks;
+      const float* beta_c = beta_s + par * C;
+
+      // ---- (1) this chunk's inputs have landed ----
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      sync_compute();
+      const float scalar_next = more ? load_scalar(ch + 1) : 0.f;  // in flight during the chunk
+      PT(0);
+
+      // ---- (2) prep: thread = (key channel c, token half) ----
+      {
+        const int c = tid & (D - 1), half = tid >> 7;
+        const int tb = half * (C / 2);
+        float G[C / 2];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int t = c0 + j;
-          if (t < ntok) {
-            if constexpr (sizeof(OT) == 2) go[(t0 + t) * v_stride + v] = __float2bfloat16_rn(__uint_as_float(x[j]));
-            else go[(t0 + t) * v_stride + v] = __uint_as_float(x[j]);
+        for (int t = 0; t < C / 2; ++t) G[t] = KDA ? Graw[(tb + t) * D + c] : gsc_s[par * C + tb + t];
+#pragma unroll
+        for (int t = 1; t < C / 2; ++t) G[t] += G[t - 1];
+        // the midpoint is the end of the first half: first-half exponents are G_t - G_m = G[t] - G[31],
+        // second-half exponents are the local running sums themselves
+        const float ref = half == 0 ? G[C / 2 - 1] : 0.f;
+        if (half == 0) fac_s[c] = ex2f((post_s[(par ^ 1) * D + c] + G[C / 2 - 1]) * LOG2E);
+        else post_s[par * D + c] = G[C / 2 - 1];  // G_C - G_m, owed to the state after this chunk
+#pragma unroll
+        for (int t4 = 0; t4 < C / 2; t4 += 4) {
+          uint32_t kht[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int t = tb + t4 + u;
+            const float kf = __bfloat162float(Kraw[t * D + c]);
+            const float qf = __bfloat162float(Qraw[t * D + c]) * a.q_scale;
+            const float d = (G[t4 + u] - ref) * LOG2E;
+            const float e1 = ex2f(d), e2 = ex2f(-d);
+            *reinterpret_cast<uint32_t *>(smem + OFF_KQ + sw128_offset(128, t, c)) = to_tf32(kf * e1);
+            *reinterpret_cast<uint32_t *>(smem + OFF_KQ + sw128_offset(128, 64 + t, c)) = to_tf32(qf * e1);
+            kht[u] = to_tf32(kf * e2);
+            *reinterpret_cast<uint32_t *>(smem + OFF_KH + sw128_offset(64, t, c)) = kht[u];
+          }
+          *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c, tb + t4)) = make_uint4(kht[0], kht[1], kht[2], kht[3]);
+        }
+      }
+      fence_smem_to_async();
+      tc_fence_before_sync();
+      mbar_arrive(&misc->rdy_prep);  // -> MMA1
+      sync_compute();                // fac_s visible; raw q/k/g consumed by everyone
+      if (more) stage_qk(ch + 1);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      PT(1);
+
+      // ---- (3) state pass: thread = (value column v, half of the channels); scale to this chunk's
+      //          midpoint and refresh the tf32 operand copy ----
+      {
+        const int cb = colh * 64;
+        uint32_t s[2][32];
+        auto fetch = [&](int c0, uint32_t(&dst)[32]) {
+          if (ch == 0) {
+            if (a.mode == DASC_REFRESH_CONTINUE) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) dst[j] = __float_as_uint(st[(c0 + j) * D + vrow]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) dst[j] = 0u;
+            }
+          } else {
+            tmem_ld32(tlane + COL_S + c0, dst);
+          }
+        };
+        fetch(cb, s[0]);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const int c0 = cb + i * 32;
+          if (ch != 0) tmem_ld_wait();
+          if (i < 1) fetch(c0 + 32, s[(i + 1) & 1]);
+          uint32_t(&cur)[32] = s[i & 1];
+          uint32_t sop[32];
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 f = *reinterpret_cast<const float4 *>(fac_s + c0 + j);
+            const float x0 = __uint_as_float(cur[j + 0]) * f.x, x1 = __uint_as_float(cur[j + 1]) * f.y;
+            const float x2 = __uint_as_float(cur[j + 2]) * f.z, x3 = __uint_as_float(cur[j + 3]) * f.w;
+            cur[j + 0] = __float_as_uint(x0); cur[j + 1] = __float_as_uint(x1);
+            cur[j + 2] = __float_as_uint(x2); cur[j + 3] = __float_as_uint(x3);
+            sop[j + 0] = to_tf32(x0); sop[j + 1] = to_tf32(x1); sop[j + 2] = to_tf32(x2); sop[j + 3] = to_tf32(x3);
+          }
+          tmem_st32(tlane + COL_S + c0, cur);
+          tmem_st32(tlane + COL_SOP + c0, sop);
+        }
+        tmem_st_wait();
+      }
+      tc_fence_before_sync();
+      mbar_arrive(&misc->rdy_state);  // -> MMA2
+      PT(2);
+
+      // ---- (4) A and P out of TMEM; T = (I + A)^-1 ----
+      wait_bar(&misc->bar_ap, par, misc, err);
+      tc_fence_after_sync();
+      PT(3);
+      {
+        uint32_t x[32];
+        const int ib = colh * 32;  // this thread's 32 columns of row `vrow`
+        tmem_ld32(tlane + COL_AP + ib, x);
+        tmem_ld_wait();
+        if (vrow < C) {
+          // lanes 0-63: row t of A = strict_lower(Kt Kh^T) * beta_t, kept in fp32 for the inverse
+          const int t = vrow;
+          const float bt = beta_c[t];
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const int i0 = ib + j;
+            float4 o;
+            o.x = (i0 + 0 < t) ? bt * __uint_as_float(x[j + 0]) : 0.f;
+            o.y = (i0 + 1 < t) ? bt * __uint_as_float(x[j + 1]) : 0.f;
+            o.z = (i0 + 2 < t) ? bt * __uint_as_float(x[j + 2]) : 0.f;
+            o.w = (i0 + 3 < t) ? bt * __uint_as_float(x[j + 3]) : 0.f;
+            *reinterpret_cast<float4 *>(Lm + t * LDX + i0) = o;
+          }
+        } else {
+          // lanes 64-127: row t of P = lower_incl_diag(Qt Kh^T), straight to its operand tile
+          const int t = vrow - C;
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const int i0 = ib + j;
+            uint4 o;
+            o.x = (i0 + 0 <= t) ? to_tf32(__uint_as_float(x[j + 0])) : 0u;
+            o.y = (i0 + 1 <= t) ? to_tf32(__uint_as_float(x[j + 1])) : 0u;
+            o.z = (i0 + 2 <= t) ? to_tf32(__uint_as_float(x[j + 2])) : 0u;
+            o.w = (i0 + 3 <= t) ? to_tf32(__uint_as_float(x[j + 3])) : 0u;
+            *reinterpret_cast<uint4 *>(smem + OFF_PM + sw128_offset(64, t, i0)) = o;
           }
         }
       }
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-  }
+      sync_compute();
+      PT(4);
+      // diagonal 16x16 blocks: thread (block b, column cc) solves (I + L_bb) x = e_cc by forward substitution
+      if (tid < C) {
+        const int b = tid >> 4, cc = tid & 15;
+        const float *Lb = Lm + (b * 16) * LDX + b * 16;
+        float x[16];
+#pragma unroll
+        for (int rr = 0; rr < 16; ++rr) {
+          float acc0 = (rr == cc) ? 1.f : 0.f, acc1 = 0.f;
+#pragma unroll
+          for (int j = 0; j + 1 < rr; j += 2) {
+            acc0 = fmaf(-Lb[rr * LDX + j], x[j], acc0);
+            acc1 = fmaf(-Lb[rr * LDX + j + 1], x[j + 1], acc1);
+          }
+          if (rr & 1) acc0 = fmaf(-Lb[rr * LDX + rr - 1], x[rr - 1], acc0);
+          x[rr] = acc0 + acc1;
+        }
+#pragma unroll
+        for (int rr = 0; rr < 16; ++rr) Xm[(b * 16 + rr) * LDX + b * 16 + cc] = x[rr];
+      }
+      sync_compute();
+      PT(5);
+      {
+        // off-diagonal blocks, X_IJ = -X_II sum_K L_IK X_KJ; Y_IJ = sum_K L_IK X_KJ is parked in the
+        // (otherwise unused) upper block (J, I) of X.  One warp per block product.
+        auto Lb = [&](int I, int J) { return Lm + (I * 16) * LDX + J * 16; };
+        auto Xb = [&](int I, int J) { return Xm + (I * 16) * LDX + J * 16; };
+        float acc[2][4];
+        auto zero = [&]() {
+#pragma unroll
+          for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        };
+        // first sub-diagonal: (1,0), (2,1), (3,2)
+        if (warp < 3) {
+          const int I = warp + 1, J = warp;
+          zero();
+          warp_mm_acc(acc, Lb(I, J), Xb(J, J), lane);
+          warp_mm_store(Xb(J, I), acc, 1.f, lane);
+          __syncwarp();
+          zero();
+          warp_mm_acc(acc, Xb(I, I), Xb(J, I), lane);
+          warp_mm_store(Xb(I, J), acc, -1.f, lane);
+        }
+        sync_compute();
+        // second sub-diagonal: (2,0), (3,1)
+        if (warp < 2) {
+          const int I = warp + 2, J = warp;
+          zero();
+          warp_mm_acc(acc, Lb(I, J), Xb(J, J), lane);
+          warp_mm_acc(acc, Lb(I, J + 1), Xb(J + 1, J), lane);
+          warp_mm_store(Xb(J, I), acc, 1.f, lane);
+          __syncwarp();
+          zero();
+          warp_mm_acc(acc, Xb(I, I), Xb(J, I), lane);
+          warp_mm_store(Xb(I, J), acc, -1.f, lane);
+        }
+        sync_compute();
+        // corner block (3,0)
+        if (warp == 0) {
+          zero();
+          warp_mm_acc(acc, Lb(3, 0), Xb(0, 0), lane);
+          warp_mm_acc(acc, Lb(3, 1), Xb(1, 0), lane);
+          warp_mm_acc(acc, Lb(3, 2), Xb(2, 0), lane);
+          warp_mm_store(Xb(0, 3), acc, 1.f, lane);
+          __syncwarp();
+          zero();
+          warp_mm_acc(acc, Xb(3, 3), Xb(0, 3), lane);
+          warp_mm_store(Xb(3, 0), acc, -1.f, lane);
+        }
+        sync_compute();
+        // T (lower triangle of X, unit diagonal) -> tf32 operand tile
+        const int t = tid >> 2, i0 = (tid & 3) * 16;
+#pragma unroll
+        for (int j = 0; j < 16; j += 4) {
+          const float4 xv = *reinterpret_cast<const float4 *>(Xm + t * LDX + i0 + j);
+          uint4 o;
+          o.x = (i0 + j + 0 <= t) ? to_tf32(xv.x) : 0u;
+          o.y = (i0 + j + 1 <= t) ? to_tf32(xv.y) : 0u;
+          o.z = (i0 + j + 2 <= t) ? to_tf32(xv.z) : 0u;
+          o.w = (i0 + j + 3 <= t) ? to_tf32(xv.w) : 0u;
+          *reinterpret_cast<uint4 *>(smem + OFF_TM + sw128_offset(64, t, i0 + j)) = o;
+        }
+      }
+      fence_smem_to_async();
+      sync_compute();  // everyone is done with L and X: the next chunk's g may land there
+      if (more) stage_g(ch + 1);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      PT(6);
 
-  // ---- final state: the factor still owed, then write back ----
-  fac_s[tid] = ex2f(prev_post * LOG2E);
-  __syncthreads();
-  tc_fence_after_sync();
-  {
-    const int v = tid;
-    const uint8_t *keep = a.row_keep + static_cast<int64_t>(layer) * a.rows_per_layer + static_cast<int64_t>(h) * D;
-    const bool merge = a.mode != DASC_REFRESH_CONTINUE;
-#pragma unroll 1
-    for (int c0 = 0; c0 < D; c0 += 32) {
-      uint32_t s[32];
-      if (n_chunks > 0) {
-        tmem_ld32(tlane + COL_S + c0, s);
+      // ---- (5) RHS^T = beta (V - R)^T, written over R^T as the tf32 A operand of MMA3 ----
+      wait_bar(&misc->bar_ro, par, misc, err);
+      tc_fence_after_sync();
+      PT(7);
+      {
+        const int tb = colh * 32;
+        uint32_t x[32];
+        tmem_ld32(tlane + COL_RO + tb, x);
         tmem_ld_wait();
-      } else {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) s[j] = 0u;  // scratch mode with an empty suffix
+        for (int j = 0; j < 32; ++j) {
+          const int t = tb + j;
+          const float vv = __bfloat162float(Vs[t * D + vrow]);
+          x[j] = to_tf32(beta_c[t] * (vv - __uint_as_float(x[j])));
+        }
+        tmem_st32(tlane + COL_RO + tb, x);
+        tmem_st_wait();
       }
+      tc_fence_before_sync();
+      mbar_arrive(&misc->rdy_rhs);  // -> MMA3 (T tile and RHS^T are ready)
+      sync_compute();               // everyone is done with V: the next chunk's tile may land
+      if (more) stage_v(ch + 1);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      PT(8);
+
+      // ---- (6) U^T rounded to tf32 in place ----
+      wait_bar(&misc->bar_u, par, misc, err);
+      tc_fence_after_sync();
+      PT(9);
+      {
+        const int tb = colh * 32;
+        uint32_t x[32];
+        tmem_ld32(tlane + COL_U + tb, x);
+        tmem_ld_wait();
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const int c = c0 + j;
-        if (!merge || !keep[c]) st[c * D + v] = __uint_as_float(s[j]) * fac_s[c];
+        for (int j = 0; j < 32; ++j) x[j] = to_tf32(__uint_as_float(x[j]));
+        tmem_st32(tlane + COL_U + tb, x);
+        tmem_st_wait();
+      }
+      tc_fence_before_sync();
+      mbar_arrive(&misc->rdy_u);  // -> MMA4, MMA5
+      PT(10);
+
+      // ---- (7) outputs of this chunk ----
+      wait_bar(&misc->bar_os, par, misc, err);
+      tc_fence_after_sync();
+      PT(11);
+      if (go) {
+        const int tb = colh * 32;
+        uint32_t x[32];
+        tmem_ld32(tlane + COL_RO + 64 + tb, x);
+        tmem_ld_wait();
+        if constexpr (sizeof(OT) == 2) {
+          // through shared memory (the Kt/Qt tile is free now) so that global stores are 16 bytes wide
+          __nv_bfloat16 *Os = reinterpret_cast<__nv_bfloat16 *>(smem + OFF_KQ);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) Os[(tb + j) * D + vrow] = __float2bfloat16_rn(__uint_as_float(x[j]));
+          sync_compute();
+          for (int i = tid; i < ntok * 16; i += NC) {
+            const int t = i >> 4, j = i & 15;
+            *reinterpret_cast<uint4 *>(reinterpret_cast<char *>(go + (t0 + t) * v_stride) + j * 16) =
+                *reinterpret_cast<const uint4 *>(smem + OFF_KQ + t * 256 + j * 16);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (tb + j < ntok) go[(t0 + tb + j) * v_stride + vrow] = __uint_as_float(x[j]);
+        }
+      }
+      store_scalar(ch + 1, scalar_next);
+      tc_fence_before_sync();
+      sync_compute();  // every thread is done with this chunk's tiles before they are rewritten
+      PT(12);
+    }
+
+    // ---- final state: the factor still owed, then write back ----
+    if (tid < D) fac_s[tid] = ex2f(post_s[((n_chunks + 1) & 1) * D + tid] * LOG2E);
+    sync_compute();
+    tc_fence_after_sync();
+    {
+      const uint8_t *keep = a.row_keep + static_cast<int64_t>(layer) * a.rows_per_layer + static_cast<int64_t>(h) * D;
+      const bool merge = a.mode != DASC_REFRESH_CONTINUE;
+#pragma unroll 1
+      for (int c0 = colh * 64; c0 < colh * 64 + 64; c0 += 32) {
+        uint32_t s[32];
+        if (n_chunks > 0) {
+          tmem_ld32(tlane + COL_S + c0, s);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) s[j] = 0u;  // scratch mode with an empty suffix
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const int c = c0 + j;
+          if (!merge || !keep[c]) st[c * D + vrow] = __uint_as_float(s[j]) * fac_s[c];
+        }
       }
     }
+    PT(13);
+    PT_DUMP;
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tm, 512);
+  if (warp == 8) tmem_dealloc(tm, 512);
 }
 
 template <bool KDA, typename OT>
