@@ -237,6 +237,40 @@ dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t l
  * Copies 4 bytes device -> host (synchronous). */
 dasc_status_t dasc_refresh_status(const void *workspace, size_t workspace_bytes);
 
+/*
+ * The paper has no counterpart to this call: it is dasc_refresh (chunked tensor-core kernel,
+ * bf16 token streams, d_k = d_v = 128) for callers that cannot hand over a workspace because
+ * they cannot allocate device memory at the point of the call.  The typical case is a serving
+ * engine whose start-up code has carved all of the GPU's memory into weights, KV cache and
+ * state pools: on the cache-hit path a cudaMalloc (or a framework allocator that may fall
+ * back to one) can fail for lack of free memory or stall the device, and no spare buffer was
+ * planned for this library.
+ *
+ * The kernel's scratch (its time-out flag) lives in a 4096-byte array that is part of the
+ * library image: every GPU that loads libdasc holds those bytes until the process exits.  A
+ * request whose scratch need (dasc_refresh_workspace_bytes) exceeds 4096 bytes is refused with
+ * DASC_ERR_WORKSPACE; shapes the chunked kernel does not take get DASC_ERR_SHAPE.  The call
+ * makes no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ * First call on a device: the library looks up the array's device address for the CURRENT
+ * device (which must be the plan's device) and remembers it.  Make that first call before any
+ * stream capture is begun, since the look-up is not a stream operation.
+ * All calls on one device share the array and it keeps the last call's contents; the call
+ * clears the flag on `cuda_stream` before the kernel runs.  Two dasc_refresh_static calls
+ * that overlap on the GPU (different streams, no ordering) race on the flag: order them, or
+ * give one of them its own workspace through dasc_refresh.
+ *
+ * Arguments are those of dasc_refresh with io_dtype fixed to bf16, algo fixed to CHUNKED and
+ * no workspace.  *scratch_out (may be NULL) receives the DEVICE address of the array, so that
+ * after synchronising the stream dasc_refresh_status(*scratch_out, 4) reports a time-out.
+ */
+dasc_status_t dasc_refresh_static(const dasc_plan_t *plan, float *state_base, int64_t layer_stride,
+                                  int64_t req_stride, const int32_t *req_idx, const void *q, const void *k,
+                                  const void *v, const float *g, const float *beta, const int32_t *cu_seqlens,
+                                  int32_t n_req, int64_t total_tokens, int32_t max_seqlen, int32_t layer_begin,
+                                  int32_t layer_end, float q_scale, void *o, int32_t o_dtype, int32_t mode,
+                                  void **scratch_out, void *cuda_stream);
+
 const char *dasc_status_string(dasc_status_t status);
 /* "major.minor.patch" of this library. */
 const char *dasc_version(void);

@@ -29,7 +29,8 @@ OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_WORKSP
 EXPORTS = (
     "dasc_plan", "dasc_plan_destroy", "dasc_plan_info", "dasc_plan_horizon", "dasc_plan_mask",
     "dasc_plan_window", "dasc_plan_layer_counts", "dasc_plan_layer_offsets", "dasc_pack", "dasc_restore",
-    "dasc_refresh_workspace_bytes", "dasc_refresh", "dasc_refresh_status", "dasc_status_string", "dasc_version",
+    "dasc_refresh_workspace_bytes", "dasc_refresh", "dasc_refresh_status", "dasc_refresh_static",
+    "dasc_status_string", "dasc_version",
 )
 
 
@@ -94,6 +95,10 @@ def lib() -> C.CDLL:
                                    C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]
         L.dasc_refresh_status.argtypes = [C.c_void_p, C.c_size_t]
+        L.dasc_refresh_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                          C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
+                                          C.c_int32, C.c_int32, C.POINTER(C.c_void_p), C.c_void_p]
         L.dasc_status_string.restype = C.c_char_p
         L.dasc_status_string.argtypes = [C.c_int]
         L.dasc_version.restype = C.c_char_p
@@ -242,3 +247,26 @@ def dasc_refresh_status(workspace: torch.Tensor | None) -> int:
     if workspace is None:
         return OK
     return int(lib().dasc_refresh_status(_ptr(workspace), int(workspace.numel() * workspace.element_size())))
+
+
+def dasc_refresh_static(plan: Plan, state: torch.Tensor, layer_stride: int, req_stride: int, req_idx: torch.Tensor,
+                        q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, g: torch.Tensor, beta: torch.Tensor,
+                        cu_seqlens: torch.Tensor, total_tokens: int, max_seqlen: int, *, layer_begin: int = 0,
+                        layer_end: int | None = None, q_scale: float = 1.0, o: torch.Tensor | None = None,
+                        mode: int = REFRESH_CONTINUE, stream=None) -> int:
+    """``dasc_refresh`` for callers that cannot allocate: no workspace argument, the kernel's scratch
+    is a fixed array inside the library.  bf16 streams and d_k = d_v = 128 only.  Returns the device
+    address of that array (for ``dasc_refresh_status`` after a synchronise).  Calls that overlap on
+    the GPU share the array and race on its time-out flag."""
+    if q.dtype != torch.bfloat16:
+        raise ValueError("dasc_refresh_static takes bf16 token streams")
+    o_io = IO_BF16 if (o is not None and o.dtype == torch.bfloat16) else IO_FP32
+    if layer_end is None:
+        layer_end = plan.info.n_layers
+    scratch = C.c_void_p()
+    _check(lib().dasc_refresh_static(plan.handle, _ptr(state), layer_stride, req_stride, _ptr(req_idx), _ptr(q),
+                                     _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(cu_seqlens),
+                                     int(cu_seqlens.numel() - 1), int(total_tokens), int(max_seqlen), layer_begin,
+                                     layer_end, float(q_scale), _ptr(o), o_io, mode, C.byref(scratch),
+                                     _stream_ptr(stream)), "dasc_refresh_static")
+    return int(scratch.value or 0)

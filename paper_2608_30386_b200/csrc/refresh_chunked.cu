@@ -706,3 +706,97 @@ int dasc_launch_refresh_chunked(const DascRefreshArgs &a, void *stream) {
   if (o_bf16) return kda ? launch<true, __nv_bfloat16>(a, stream) : launch<false, __nv_bfloat16>(a, stream);
   return kda ? launch<true, float>(a, stream) : launch<false, float>(a, stream);
 }
+
+// ---------------------------------------------------------------------------------------------
+// dasc_refresh_static: the chunked refresh without any caller-provided workspace.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// Scratch of the static variant.  It lives in the library image: every GPU that loads libdasc
+// holds these bytes until the process exits.  In host code the name below is only a handle; the
+// device address is obtained once per device with cudaGetSymbolAddress.
+constexpr size_t kStaticScratchBytes = 4096;
+static __device__ __align__(256) unsigned char g_refresh_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_addr[kMaxDevices] = {};  // device address per CUDA device, filled on first use
+
+// Device address of the static scratch on the CURRENT device; resolves it on the first call.
+cudaError_t static_scratch_address(void **out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  void *p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    e = cudaGetSymbolAddress(&p, g_refresh_static_scratch);
+    if (e != cudaSuccess) return e;
+    __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);  // racing first calls store the same value
+  }
+  *out = p;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" dasc_status_t dasc_refresh_static(const dasc_plan_t *plan, float *state_base, int64_t layer_stride,
+                                             int64_t req_stride, const int32_t *req_idx, const void *q, const void *k,
+                                             const void *v, const float *g, const float *beta,
+                                             const int32_t *cu_seqlens, int32_t n_req, int64_t total_tokens,
+                                             int32_t max_seqlen, int32_t layer_begin, int32_t layer_end, float q_scale,
+                                             void *o, int32_t o_dtype, int32_t mode, void **scratch_out,
+                                             void *cuda_stream) {
+  if (scratch_out) *scratch_out = nullptr;
+  if (!plan || plan->info.device < 0) return DASC_ERR_INVALID_ARG;
+  if (n_req < 0 || total_tokens < 0 || max_seqlen < 0) return DASC_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_end < layer_begin || layer_end > plan->info.n_layers) return DASC_ERR_INVALID_ARG;
+  if (o && o_dtype != DASC_IO_BF16 && o_dtype != DASC_IO_FP32) return DASC_ERR_INVALID_ARG;
+  if (mode != DASC_REFRESH_CONTINUE && mode != DASC_REFRESH_SCRATCH_MERGE_LOCAL) return DASC_ERR_INVALID_ARG;
+  if (plan->info.d_k != D || plan->info.d_v != D) return DASC_ERR_SHAPE;  // the chunked kernel's shape
+  // The scratch this request would need from a caller must fit the static array.
+  const size_t need = dasc_refresh_chunked_workspace_bytes(n_req, layer_end - layer_begin, plan->info.n_v_heads);
+  if (need > kStaticScratchBytes) return DASC_ERR_WORKSPACE;
+  void *scratch = nullptr;
+  if (static_scratch_address(&scratch) != cudaSuccess) return DASC_ERR_CUDA;
+  if (scratch_out) *scratch_out = scratch;
+  if (n_req == 0 || layer_end == layer_begin || total_tokens == 0) return DASC_OK;
+  if (!state_base || !req_idx || !q || !k || !v || !g || !beta || !cu_seqlens) return DASC_ERR_INVALID_ARG;
+  auto misaligned = [](const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+  if (misaligned(state_base) || misaligned(q) || misaligned(k) || misaligned(v) || misaligned(g) || (o && misaligned(o)))
+    return DASC_ERR_INVALID_ARG;
+  if (layer_stride < 0 || req_stride < 0 || layer_stride % 4 || req_stride % 4) return DASC_ERR_INVALID_ARG;
+
+  DascRefreshArgs a{};
+  a.kind = plan->info.kind;
+  a.H_v = plan->info.n_v_heads;
+  a.H_k = plan->info.n_k_heads;
+  a.d_k = plan->info.d_k;
+  a.d_v = plan->info.d_v;
+  a.state = state_base;
+  a.layer_stride = layer_stride;
+  a.req_stride = req_stride;
+  a.req_idx = req_idx;
+  a.q = q;
+  a.k = k;
+  a.v = v;
+  a.io_bf16 = 1;
+  a.g = g;
+  a.beta = beta;
+  a.cu_seqlens = cu_seqlens;
+  a.n_req = n_req;
+  a.total_tokens = total_tokens;
+  a.max_seqlen = max_seqlen;
+  a.layer_begin = layer_begin;
+  a.n_layers_in_call = layer_end - layer_begin;
+  a.q_scale = q_scale;
+  a.o = o;
+  a.o_bf16 = o_dtype == DASC_IO_BF16;
+  a.mode = mode;
+  a.row_keep = plan->d_row_keep;
+  a.rows_per_layer = plan->rows_per_layer;
+  a.workspace = scratch;  // the launcher clears the time-out flag (first word) on the stream
+  a.workspace_bytes = kStaticScratchBytes;
+  const int e = dasc_launch_refresh_chunked(a, cuda_stream);
+  if (e == -1) return DASC_ERR_SHAPE;
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
