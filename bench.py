@@ -371,9 +371,15 @@ def main():
                  "traffic": None, "peak_source": src, "frac_of_8TBps_nominal": pack_gbs / 8000.0},
         "restore": {"bound": "hbm", "achieved": restore_gbs, "peak": hbm, "unit": "GB/s", "frac": restore_gbs / hbm,
                     "traffic": None, "peak_source": src, "frac_of_8TBps_nominal": restore_gbs / 8000.0},
+        # By the arithmetic (about 100 flop per byte, below the ridge) HBM is the ceiling of the refresh;
+        # the tensor-pipe figures beside it: tf32 flops the chunked kernel issues (163,840 per token-head)
+        # against the tf32 peak taken as 0.489 x the measured sustained bf16 peak (nominal 1.1 : 2.25).
         "refresh": {"bound": "hbm", "achieved": refresh_gbs, "peak": hbm, "unit": "GB/s", "frac": refresh_gbs / hbm,
                     "traffic": None, "peak_source": src, "tflops_min_form": refresh_tflops,
-                    "frac_of_bf16_tensor_sustained": refresh_tflops / tf, "frac_of_fp32_alu": refresh_tflops / alu_tflops},
+                    "frac_of_fp32_alu": refresh_tflops / alu_tflops,
+                    "tflops_tf32_issued": token_heads * 163840 / (t_refresh * 1e-3) / 1e12,
+                    "tf32_peak": 0.489 * tf,
+                    "frac_of_tf32_tensor": token_heads * 163840 / (t_refresh * 1e-3) / 1e12 / (0.489 * tf)},
     }
     dominant = max((("pack", t_pack), ("restore", t_restore), ("refresh", t_refresh)), key=lambda x: x[1])[0]
     roofline = dict(rl[dominant])

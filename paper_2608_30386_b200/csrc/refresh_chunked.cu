@@ -83,7 +83,7 @@ constexpr uint32_t kMaxPolls = 1u << 22;
 
 struct Misc {
   // tensor core -> compute warps (one tcgen05.commit each per chunk)
-  uint64_t bar_ap, bar_ro, bar_u, bar_os;
+  uint64_t bar_ap, bar_ro, bar_u, bar_o, bar_s;
   // compute warps -> issuing warp (256 arrivals each per chunk)
   uint64_t rdy_prep, rdy_state, rdy_rhs, rdy_u;
   uint32_t tmem_base;
@@ -196,7 +196,8 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
     mbar_init(&misc->bar_ap, 1);
     mbar_init(&misc->bar_ro, 1);
     mbar_init(&misc->bar_u, 1);
-    mbar_init(&misc->bar_os, 1);
+    mbar_init(&misc->bar_o, 1);
+    mbar_init(&misc->bar_s, 1);
     mbar_init(&misc->rdy_prep, NC);
     mbar_init(&misc->rdy_state, NC);
     mbar_init(&misc->rdy_rhs, NC);
@@ -252,12 +253,15 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
       __syncwarp();
       if (lane == 0) {
         tc_fence_after_sync();
+        // RHS^T is given as a tf32 pair (high part over R^T, low part in the A|P columns)
 #pragma unroll
-        for (int kb = 0; kb < 2; ++kb)
+        for (int part = 0; part < 2; ++part)
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            mma_ts(tm + COL_U, tm + COL_RO + kb * 32 + j * 8, desc_kmajor(sbase + OFF_TM + kb * (64 * 128) + j * 32),
-                   ID_M128_N64, (kb | j) != 0);
+          for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              mma_ts(tm + COL_U, tm + (part == 0 ? COL_RO : COL_AP) + kb * 32 + j * 8,
+                     desc_kmajor(sbase + OFF_TM + kb * (64 * 128) + j * 32), ID_M128_N64, (part | kb | j) != 0);
         mma_commit(&misc->bar_u);
       }
       // MMA4: O^T += U^T P^T;  MMA5: S'^T += U^T Kh
@@ -265,6 +269,8 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
       __syncwarp();
       if (lane == 0) {
         tc_fence_after_sync();
+        // U^T is given as a tf32 pair (high part in place, low part over the consumed RHS^T columns)
+        // (the outputs take the high part only: their error budget does not need the low part)
         if (go) {
 #pragma unroll
           for (int kb = 0; kb < 2; ++kb)
@@ -273,13 +279,16 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
               mma_ts(tm + COL_RO + 64, tm + COL_U + kb * 32 + j * 8,
                      desc_kmajor(sbase + OFF_PM + kb * (64 * 128) + j * 32), ID_M128_N64, true);
         }
+        mma_commit(&misc->bar_o);
 #pragma unroll
-        for (int kb = 0; kb < 2; ++kb)
+        for (int part = 0; part < 2; ++part)
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            mma_ts(tm + COL_S, tm + COL_U + kb * 32 + j * 8, desc_kmajor(sbase + OFF_KHT + kb * (128 * 128) + j * 32),
-                   ID_M128_N128, true);
-        mma_commit(&misc->bar_os);
+          for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              mma_ts(tm + COL_S, tm + (part == 0 ? COL_U : COL_RO) + kb * 32 + j * 8,
+                     desc_kmajor(sbase + OFF_KHT + kb * (128 * 128) + j * 32), ID_M128_N128, true);
+        mma_commit(&misc->bar_s);
       }
       __syncwarp();
     }
@@ -351,7 +360,9 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
       const bool more = ch + 1 < n_chunks;
       const float* beta_c = beta_s + par * C;
 
-      // ---- (1) this chunk's inputs have landed ----
+      // ---- (1) this chunk's inputs have landed; the previous chunk's state update is complete ----
+      if (ch > 0) wait_bar(&misc->bar_s, par ^ 1, misc, err);
+      tc_fence_after_sync();
       asm volatile("cp.async.wait_all;" ::: "memory");
       sync_compute();
       const float scalar_next = more ? load_scalar(ch + 1) : 0.f;  // in flight during the chunk
@@ -577,16 +588,19 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
       PT(7);
       {
         const int tb = colh * 32;
-        uint32_t x[32];
+        uint32_t x[32], lo[32];
         tmem_ld32(tlane + COL_RO + tb, x);
         tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const int t = tb + j;
           const float vv = __bfloat162float(Vs[t * D + vrow]);
-          x[j] = to_tf32(beta_c[t] * (vv - __uint_as_float(x[j])));
+          const float rhs = beta_c[t] * (vv - __uint_as_float(x[j]));
+          x[j] = to_tf32(rhs);                                  // high part
+          lo[j] = to_tf32(rhs - __uint_as_float(x[j]));         // what the high part lost
         }
         tmem_st32(tlane + COL_RO + tb, x);
+        tmem_st32(tlane + COL_AP + tb, lo);  // the A|P columns were consumed in step (4)
         tmem_st_wait();
       }
       tc_fence_before_sync();
@@ -602,12 +616,17 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
       PT(9);
       {
         const int tb = colh * 32;
-        uint32_t x[32];
+        uint32_t x[32], lo[32];
         tmem_ld32(tlane + COL_U + tb, x);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) x[j] = to_tf32(__uint_as_float(x[j]));
+        for (int j = 0; j < 32; ++j) {
+          const float u = __uint_as_float(x[j]);
+          x[j] = to_tf32(u);
+          lo[j] = to_tf32(u - __uint_as_float(x[j]));
+        }
         tmem_st32(tlane + COL_U + tb, x);
+        tmem_st32(tlane + COL_RO + tb, lo);  // RHS^T has been consumed by MMA3
         tmem_st_wait();
       }
       tc_fence_before_sync();
@@ -615,7 +634,7 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
       PT(10);
 
       // ---- (7) outputs of this chunk ----
-      wait_bar(&misc->bar_os, par, misc, err);
+      wait_bar(&misc->bar_o, par, misc, err);
       tc_fence_after_sync();
       PT(11);
       if (go) {
@@ -647,6 +666,7 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
     }
 
     // ---- final state: the factor still owed, then write back ----
+    if (n_chunks > 0) wait_bar(&misc->bar_s, (n_chunks - 1) & 1, misc, err);
     if (tid < D) fac_s[tid] = ex2f(post_s[((n_chunks + 1) & 1) * D + tid] * LOG2E);
     sync_compute();
     tc_fence_after_sync();
