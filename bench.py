@@ -2,16 +2,23 @@
 """Benchmark of the DASC hot path on B200: one step = pack -> restore (zero-fill) ->
 suffix refresh over one batch of synthetic state checkpoints.
 
-Workload (N=1): the serving-scale KDA configuration -- 24 KDA layers x 32 heads x
-128x128 fp32 states (2 MiB per layer and request), 64 requests, per-channel decay rates
-log-uniform in [1e-3, 1] (seed 1), keep ratio 0.38 per layer -- followed by a refresh of
-a 256-token bf16 suffix per request.  Inputs are far larger than L2, so no flush is needed.
+Default workload (N=1, the one the driver times): the serving-scale KDA configuration --
+24 KDA layers x 32 heads x 128x128 fp32 states (2 MiB per layer and request), 64 requests,
+per-channel decay rates log-uniform in [1e-3, 1] (seed 1), keep ratio 0.38 per layer --
+followed by a refresh of a 256-token bf16 suffix per request.  Inputs are far larger than
+L2, so no flush is needed.
 
 Prints ONE JSON line.  `value` is pack+restore algorithmic GB/s (bytes the two copies must
 move / their device time); refresh throughput, per-kernel rooflines, the end-to-end leg
 (host buffers, copies timed) and the CPU oracle baseline ride along in the same line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Other configurations (not the default line; used to fill the results table):
+    --config 2            GDN head-wise, 36 layers, 32/16 heads, 128 requests, keep 0.5
+    --config 3 --suffix S aggressive KDA, keep 0.2, batch 32, suffix 256 / 1024 / 4096
+    --config 4            mixed serving trace: pack on one stream, restore+refresh on another
+    --keep R              keep ratio of the sweep {0.25, 0.38, 0.5, 1.0} for --config 1
 """
 from __future__ import annotations
 
@@ -30,9 +37,21 @@ sys.path.insert(0, ROOT)
 import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
-WORKLOAD = "kda_serving_24x32x128x128_fp32_64req_keep0.38_suffix256_bf16"
-L, H, D, N_REQ, KEEP, SUFFIX, SEED = 24, 32, 128, 64, 0.38, 256, 1
+D = 128
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+TF32_OVER_BF16 = 0.489        # nominal dense 1.1 : 2.25
+CHUNKED_FLOPS_PER_TOKEN_HEAD = 163840   # tf32 flops the chunked kernel issues per (token, head)
+
+CONFIGS = {
+    1: dict(name="kda_serving", kind="KDA", L=24, H_v=32, H_k=32, n_req=64, keep=0.38, rate_lo=1e-3, suffix=256, seed=1),
+    2: dict(name="gdn_headwise", kind="GDN", L=36, H_v=32, H_k=16, n_req=128, keep=0.5, rate_lo=1e-4, suffix=256, seed=2),
+    3: dict(name="kda_aggressive", kind="KDA", L=24, H_v=32, H_k=32, n_req=32, keep=0.2, rate_lo=1e-3, suffix=256, seed=3),
+    4: dict(name="mixed_trace", kind="KDA", L=24, H_v=32, H_k=32, n_req=64, keep=0.38, rate_lo=1e-3, suffix=1024, seed=4),
+}
+
+
+def workload_name(c):
+    return (f"{c['name']}_{c['L']}x{c['H_v']}x{D}x{D}_fp32_{c['n_req']}req_keep{c['keep']}_suffix{c['suffix']}_bf16")
 
 
 def peaks():
@@ -102,103 +121,131 @@ class ClockSampler:
 # CPU oracle leg (the reported baseline and the whole of --impl reference)
 # ----------------------------------------------------------------------------------------------
 
-def oracle_leg(sample_req=4, sample_units=64):
+def oracle_leg(c, sample_req=4, sample_units=64):
     """Times the fp64 oracle, as it stands, on a bounded sample of the same workload."""
     import oracle
     from paper_2608_30386_b200 import synth
 
-    gen = synth.generator(SEED)
-    rates = synth.decay_rates(gen, L, H, D, 1e-3, 1.0)
+    kda = c["kind"] == "KDA"
+    okind = oracle.KDA if kda else oracle.GDN
+    L, H_v, H_k = c["L"], c["H_v"], c["H_k"]
+    uph = D if kda else 1
+    gen = synth.generator(c["seed"])
+    rates = synth.decay_rates(gen, L, H_v, uph, c["rate_lo"], 1.0)
     A_log, dt = synth.decay_params(rates)
-    oplan = oracle.plan(oracle.KDA, L, H, D, A_log.numpy(), dt.numpy(), sel=oracle.SEL_TOP_RATIO, keep_ratio=KEEP,
-                        scope=oracle.SCOPE_LAYER, unit_bytes=D * 4)
-    dense = H * D * D
+    unit_words = D if kda else D * D
+    oplan = oracle.plan(okind, L, H_v, uph, A_log.numpy(), dt.numpy(), sel=oracle.SEL_TOP_RATIO,
+                        keep_ratio=c["keep"], scope=oracle.SCOPE_LAYER, unit_bytes=unit_words * 4)
+    dense = H_v * D * D
     state = synth.states(gen, (sample_req, L, dense)).numpy()
-    slot = oplan.sum_r * D
+    slot = oplan.sum_r * unit_words
     pool = np.zeros((sample_req, slot), np.float32)
     out = np.empty_like(state)
     ids = np.arange(sample_req, dtype=np.int32)
     t0 = time.perf_counter()
-    oracle.pack(oplan.mask, D, state, dense, L * dense, ids, pool, slot, ids)
+    oracle.pack(oplan.mask, unit_words, state, dense, L * dense, ids, pool, slot, ids)
     t1 = time.perf_counter()
-    oracle.restore(oplan.mask, D, pool, slot, ids, out, dense, L * dense, ids)
+    oracle.restore(oplan.mask, unit_words, pool, slot, ids, out, dense, L * dense, ids)
     t2 = time.perf_counter()
     pack_bytes = 2 * sample_req * slot * 4
     restore_bytes = sample_req * (slot + L * dense) * 4
-    # refresh sample: `sample_units` (request, layer, head) units = 2 layers x 32 heads of one request
-    Ls = max(1, sample_units // H)
-    streams = synth.token_streams(gen, synth.KDA, Ls, SUFFIX, H, H, D, D, rates[:Ls])
-    st = synth.states(gen, (1, Ls, H, D, D)).numpy()
+    # refresh sample: whole layers of one request (sample_units (request, layer, head) units), 256 tokens
+    Ls = max(1, sample_units // H_v)
+    n_tok = min(c["suffix"], 256)
+    streams = synth.token_streams(gen, synth.KDA if kda else synth.GDN, Ls, n_tok, H_v, H_k, D, D, rates[:Ls])
+    st = synth.states(gen, (1, Ls, H_v, D, D)).numpy()
     threads = oracle.max_threads()
     t3 = time.perf_counter()
-    oracle.refresh(oracle.KDA, Ls, H, H, D, D, st, dense, Ls * dense, [0], synth.bf16_bits(streams.q),
+    oracle.refresh(okind, Ls, H_v, H_k, D, D, st, dense, Ls * dense, [0], synth.bf16_bits(streams.q),
                    synth.bf16_bits(streams.k), synth.bf16_bits(streams.v), streams.g.numpy(), streams.beta.numpy(),
-                   [0, SUFFIX], n_threads=threads)
+                   [0, n_tok], n_threads=threads)
     t4 = time.perf_counter()
-    token_heads = Ls * H * SUFFIX
-    # tokens/s of the full model (all L layers and H heads per token), extrapolated from the sampled units
-    refresh_tokens_per_s = token_heads / (t4 - t3) / (L * H)
+    token_heads = Ls * H_v * n_tok
     return {
         "value": (pack_bytes + restore_bytes) / (t2 - t0) / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
-        "sample": (f"pack+restore of {sample_req} of {N_REQ} requests (single thread); refresh of {Ls * H} of "
-                   f"{N_REQ * L * H} (request,layer,head) units x {SUFFIX} tokens on {threads} threads"),
+        "sample": (f"pack+restore of {sample_req} of {c['n_req']} requests (one thread); refresh of {Ls * H_v} of "
+                   f"{c['n_req'] * L * H_v} (request,layer,head) units x {n_tok} tokens on {threads} threads"),
         "pack_GBps": pack_bytes / (t1 - t0) / 1e9, "restore_GBps": restore_bytes / (t2 - t1) / 1e9,
-        "refresh_tokens_per_s": refresh_tokens_per_s, "refresh_token_heads_per_s": token_heads / (t4 - t3),
+        # tokens/s of the full model (all layers and heads per token), extrapolated from the sampled units
+        "refresh_tokens_per_s": token_heads / (t4 - t3) / (L * H_v),
+        "refresh_token_heads_per_s": token_heads / (t4 - t3),
         "seconds": t4 - t0,
     }
 
 
-def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+def run_reference(args, c):
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    vals = []
-    leg = None
+    vals, leg = [], None
     for i in range(args.warmup + args.steps):
-        leg = oracle_leg(sample_req=2, sample_units=32)
+        leg = oracle_leg(c, sample_req=2, sample_units=32)
         if i >= args.warmup:
             vals.append(leg)
     value = statistics.mean(v["value"] for v in vals)
     sec = statistics.mean(v["seconds"] for v in vals)
-    line = {
+    print(json.dumps({
         "impl": "reference", "metric": "pack_restore_GBps", "value": value, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "note": "CPU oracle on a bounded sample of the workload per step"},
+        "config": {"workload": workload_name(c), "note": "CPU oracle on a bounded sample of the workload per step"},
         "refresh_tokens_per_s": statistics.mean(v["refresh_tokens_per_s"] for v in vals),
-        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": leg["cores"], "kind": "oracle",
-                         "sample": leg["sample"]},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": leg["cores"], "kind": "oracle", "sample": leg["sample"]},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
-    }
-    print(json.dumps(line))
+    }))
 
 
 # ----------------------------------------------------------------------------------------------
 # GPU legs
 # ----------------------------------------------------------------------------------------------
 
+def build_plan(c, device):
+    import paper_2608_30386_b200 as dasc
+    from paper_2608_30386_b200 import synth
+    kda = c["kind"] == "KDA"
+    gen = synth.generator(c["seed"])
+    rates = synth.decay_rates(gen, c["L"], c["H_v"], D if kda else 1, c["rate_lo"], 1.0)
+    A_log, dt = synth.decay_params(rates)
+    plan = dasc.dasc_plan(dasc.KDA if kda else dasc.GDN, c["L"], c["H_v"], c["H_k"], D, D, A_log.numpy(), dt.numpy(),
+                          sel=dasc.SEL_TOP_RATIO, scope=dasc.SCOPE_LAYER, keep_ratio=c["keep"], device=device)
+    return plan, rates, gen
+
+
+def token_bytes_per_head(kda: bool, H_v: int, H_k: int) -> float:
+    """Algorithmic bytes per (token, value head): q + k (shared by H_v/H_k value heads) + v bf16, g fp32, beta, o bf16."""
+    share = H_k / H_v
+    return 2 * D * 2 * share + D * 2 + (D * 4 if kda else 4) + 4 + D * 2
+
+
 def main():
-    global N_REQ, SUFFIX, KEEP, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="dasc", choices=["dasc", "reference"])
     ap.add_argument("--algo", default="auto", choices=["auto", "sequential", "chunked"])
+    ap.add_argument("--config", type=int, default=1, choices=sorted(CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--requests", type=int, default=N_REQ, help="profiling only: shrink the batch")
-    ap.add_argument("--suffix", type=int, default=SUFFIX, help="profiling only: shrink the refresh suffix")
-    ap.add_argument("--keep", type=float, default=KEEP, help="keep ratio (0.25, 0.38, 0.5, 1.0 in the sweep)")
+    ap.add_argument("--requests", type=int, default=None, help="profiling only: shrink the batch")
+    ap.add_argument("--suffix", type=int, default=None, help="refresh suffix length (config 3: 256, 1024, 4096)")
+    ap.add_argument("--keep", type=float, default=None, help="keep ratio (0.25, 0.38, 0.5, 1.0 in the sweep)")
+    ap.add_argument("--layer-group", type=int, default=None, help="layers of token streams resident at once")
     args = ap.parse_args()
-    if (args.requests, args.suffix, args.keep) != (N_REQ, SUFFIX, KEEP):
-        N_REQ, SUFFIX, KEEP = args.requests, args.suffix, args.keep
-        WORKLOAD = f"kda_24x32x128x128_fp32_{N_REQ}req_keep{KEEP}_suffix{SUFFIX}_bf16"
+    c = dict(CONFIGS[args.config])
+    if args.requests is not None:
+        c["n_req"] = args.requests
+    if args.suffix is not None:
+        c["suffix"] = args.suffix
+    if args.keep is not None:
+        c["keep"] = args.keep
     if args.impl == "reference":
-        run_reference(args)
+        run_reference(args, c)
         return
     args.warmup = max(args.warmup, 3)
+    if args.config == 4:
+        run_mixed_trace(args, c)
+        return
 
     import paper_2608_30386_b200 as dasc
     from paper_2608_30386_b200 import synth
@@ -215,16 +262,14 @@ def main():
 
     algo = {"auto": dasc.ALGO_AUTO, "sequential": dasc.ALGO_SEQUENTIAL, "chunked": dasc.ALGO_CHUNKED}[args.algo]
     pk = peaks()
+    kda = c["kind"] == "KDA"
+    L, H_v, H_k, N_REQ, SUFFIX = c["L"], c["H_v"], c["H_k"], c["n_req"], c["suffix"]
 
     # ---- plan and inputs (replicas: every rank holds the same shape of work, its own seed) ----
-    gen = synth.generator(SEED)
-    rates = synth.decay_rates(gen, L, H, D, 1e-3, 1.0)
-    A_log, dt = synth.decay_params(rates)
-    plan = dasc.dasc_plan(dasc.KDA, L, H, H, D, D, A_log.numpy(), dt.numpy(), sel=dasc.SEL_TOP_RATIO,
-                          scope=dasc.SCOPE_LAYER, keep_ratio=KEEP, device=local)
-    dense = H * D * D
+    plan, rates, gen = build_plan(c, local)
+    dense = H_v * D * D
     layer_stride, req_stride = N_REQ * dense, dense          # layer-major active-state pool
-    dgen = synth.generator(SEED + 1000 * rank, dev)
+    dgen = synth.generator(c["seed"] + 1000 * rank, dev)
     state = synth.states(dgen, (L, N_REQ, dense), dev)
     active = torch.empty_like(state)
     slot = int(plan.slot_floats)
@@ -232,24 +277,27 @@ def main():
     ids = torch.arange(N_REQ, dtype=torch.int32, device=dev)
     slots = torch.randperm(N_REQ, generator=gen).to(torch.int32).to(dev)
     T = N_REQ * SUFFIX
-    streams = []
-    for l in range(L):                                       # per layer, to bound the generator's temporaries
-        s = synth.token_streams(dgen, synth.KDA, 1, T, H, H, D, D, rates[l:l + 1], device=dev)
-        streams.append(s)
-    q = torch.cat([s.q for s in streams]); k = torch.cat([s.k for s in streams]); v = torch.cat([s.v for s in streams])
-    g = torch.cat([s.g for s in streams]); beta = torch.cat([s.beta for s in streams])
-    del streams
-    o = torch.empty((L, T, H, D), dtype=torch.bfloat16, device=dev)
+    # token streams: `group` layers resident at once; when that is fewer than all layers the same
+    # buffers are replayed for every layer group (bounds memory; the work per group is identical)
+    per_layer = T * (2 * H_k * D * 2 + 2 * H_v * D * 2 + H_v * (D if kda else 1) * 4 + H_v * 4)
+    group = args.layer_group or max(1, min(L, int(40e9 // per_layer)))
+    while L % group:
+        group -= 1
+    skind = synth.KDA if kda else synth.GDN
+    parts = [synth.token_streams(dgen, skind, 1, T, H_v, H_k, D, D, rates[l:l + 1], device=dev) for l in range(group)]
+    q, k, v, g, beta = (torch.cat([getattr(p, f) for p in parts]) for f in ("q", "k", "v", "g", "beta"))
+    del parts
+    o = torch.empty((group, T, H_v, D), dtype=torch.bfloat16, device=dev)
     cu = synth.uniform_cu_seqlens(N_REQ, SUFFIX).to(dev)
-    ws_bytes = dasc.dasc_refresh_workspace_bytes(plan, N_REQ, L, algo)
+    ws_bytes = dasc.dasc_refresh_workspace_bytes(plan, N_REQ, group, algo)
     ws = torch.zeros(max(ws_bytes, 256), dtype=torch.uint8, device=dev) if ws_bytes else None
 
     pack_bytes = 2 * N_REQ * slot * 4
     restore_bytes = N_REQ * (slot + L * dense) * 4
-    token_heads = N_REQ * L * H * SUFFIX
-    # refresh algorithmic bytes per (token, head): q + k + v bf16, g fp32, beta, o bf16; plus the state in and out
-    refresh_bytes = token_heads * (3 * D * 2 + D * 4 + 4 + D * 2) + 2 * N_REQ * L * dense * 4
+    token_heads = N_REQ * L * H_v * SUFFIX
+    refresh_bytes = token_heads * token_bytes_per_head(kda, H_v, H_k) + 2 * N_REQ * L * dense * 4  # + state in and out
     refresh_flops_min = token_heads * 7 * D * D              # token-by-token recurrence, incl. decay and read-out
+    n_groups = L // group
 
     stream = torch.cuda.current_stream()
 
@@ -262,8 +310,9 @@ def main():
         dasc.dasc_restore(plan, pool, slots, active, layer_stride, req_stride, ids)
         if ev:
             ev[2].record(stream)
-        dasc.dasc_refresh(plan, active, layer_stride, req_stride, ids, q, k, v, g, beta, cu, T, SUFFIX, o=o,
-                          algo=algo, workspace=ws)
+        for gi in range(n_groups):
+            dasc.dasc_refresh(plan, active, layer_stride, req_stride, ids, q, k, v, g, beta, cu, T, SUFFIX,
+                              layer_begin=gi * group, layer_end=(gi + 1) * group, o=o, algo=algo, workspace=ws)
         if ev:
             ev[3].record(stream)
 
@@ -301,17 +350,18 @@ def main():
     if not args.no_e2e:
         n_e = min(16, N_REQ)                                 # requests per e2e step (bounded pinned memory)
         Te = n_e * SUFFIX
+        ge = min(group, 6)                                   # layers of token streams copied per refresh call
         h_state = torch.empty((L, n_e, dense), dtype=torch.float32).pin_memory()
         h_state.copy_(state[:, :n_e])
-        host_streams = [x[:, :Te].contiguous().cpu().pin_memory() for x in (q, k, v, g, beta)]
+        host_streams = [x[:ge, :Te].contiguous().cpu().pin_memory() for x in (q, k, v, g, beta)]
         h_pool = torch.empty((n_e, slot), dtype=torch.float32).pin_memory()
         h_out = torch.empty((L, n_e, dense), dtype=torch.float32).pin_memory()
-        h_o = torch.empty((L, Te, H, D), dtype=torch.bfloat16).pin_memory()
+        h_o = torch.empty((ge, Te, H_v, D), dtype=torch.bfloat16).pin_memory()
         d_state = torch.empty((L, n_e, dense), device=dev)
         d_active = torch.empty_like(d_state)
         d_pool = torch.empty((n_e, slot), device=dev)
         d_streams = [torch.empty(x.shape, dtype=x.dtype, device=dev) for x in host_streams]
-        d_o = torch.empty((L, Te, H, D), dtype=torch.bfloat16, device=dev)
+        d_o = torch.empty((ge, Te, H_v, D), dtype=torch.bfloat16, device=dev)
         cu_e = synth.uniform_cu_seqlens(n_e, SUFFIX).to(dev)
         ids_e = torch.arange(n_e, dtype=torch.int32, device=dev)
         ls_e = n_e * dense
@@ -323,12 +373,13 @@ def main():
             dasc.dasc_restore(plan, d_pool, ids_e, d_active, ls_e, dense, ids_e)
             h_pool.copy_(d_pool, non_blocking=True)
             ev[1].record(stream)
-            for dst, src in zip(d_streams, host_streams):
-                dst.copy_(src, non_blocking=True)
-            dasc.dasc_refresh(plan, d_active, ls_e, dense, ids_e, *d_streams, cu_e, Te, SUFFIX, o=d_o, algo=algo,
-                              workspace=ws)
+            for gi in range(L // ge):                        # every layer group: its streams in, its outputs out
+                for dst, src in zip(d_streams, host_streams):
+                    dst.copy_(src, non_blocking=True)
+                dasc.dasc_refresh(plan, d_active, ls_e, dense, ids_e, *d_streams, cu_e, Te, SUFFIX,
+                                  layer_begin=gi * ge, layer_end=(gi + 1) * ge, o=d_o, algo=algo, workspace=ws)
+                h_o.copy_(d_o, non_blocking=True)
             h_out.copy_(d_active, non_blocking=True)
-            h_o.copy_(d_o, non_blocking=True)
             ev[2].record(stream)
 
         n_steps_e = max(2, min(args.steps, 3))
@@ -345,8 +396,8 @@ def main():
             dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         t_copy, t_ref = tt.tolist()
         e_bytes = (2 * n_e * slot + n_e * (slot + L * dense)) * 4
-        h2d = h_state.numel() * 4 + sum(x.numel() * x.element_size() for x in host_streams)
-        d2h = h_pool.numel() * 4 + h_out.numel() * 4 + h_o.numel() * 2
+        h2d = h_state.numel() * 4 + (L // ge) * sum(x.numel() * x.element_size() for x in host_streams)
+        d2h = h_pool.numel() * 4 + h_out.numel() * 4 + (L // ge) * h_o.numel() * 2
         e2e = {"value": world * e_bytes / (t_copy * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "requests_per_step": n_e,
                "refresh_tokens_per_s": world * Te / (t_ref * 1e-3), "ms_pack_restore": t_copy, "ms_refresh": t_ref,
@@ -366,20 +417,19 @@ def main():
     # fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop x max SM clock
     alu_tflops = 148 * 128 * 2 * float(pk.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
     refresh_tflops = refresh_flops_min / (t_refresh * 1e-3) / 1e12
+    tf32_issued = token_heads * CHUNKED_FLOPS_PER_TOKEN_HEAD / (t_refresh * 1e-3) / 1e12
     rl = {
         "pack": {"bound": "hbm", "achieved": pack_gbs, "peak": hbm, "unit": "GB/s", "frac": pack_gbs / hbm,
                  "traffic": None, "peak_source": src, "frac_of_8TBps_nominal": pack_gbs / 8000.0},
         "restore": {"bound": "hbm", "achieved": restore_gbs, "peak": hbm, "unit": "GB/s", "frac": restore_gbs / hbm,
                     "traffic": None, "peak_source": src, "frac_of_8TBps_nominal": restore_gbs / 8000.0},
         # By the arithmetic (about 100 flop per byte, below the ridge) HBM is the ceiling of the refresh;
-        # the tensor-pipe figures beside it: tf32 flops the chunked kernel issues (163,840 per token-head)
-        # against the tf32 peak taken as 0.489 x the measured sustained bf16 peak (nominal 1.1 : 2.25).
+        # the tensor-pipe figures beside it: tf32 flops the chunked kernel issues against the tf32 peak
+        # taken as 0.489 x the measured sustained bf16 peak (nominal 1.1 : 2.25).
         "refresh": {"bound": "hbm", "achieved": refresh_gbs, "peak": hbm, "unit": "GB/s", "frac": refresh_gbs / hbm,
                     "traffic": None, "peak_source": src, "tflops_min_form": refresh_tflops,
-                    "frac_of_fp32_alu": refresh_tflops / alu_tflops,
-                    "tflops_tf32_issued": token_heads * 163840 / (t_refresh * 1e-3) / 1e12,
-                    "tf32_peak": 0.489 * tf,
-                    "frac_of_tf32_tensor": token_heads * 163840 / (t_refresh * 1e-3) / 1e12 / (0.489 * tf)},
+                    "frac_of_fp32_alu": refresh_tflops / alu_tflops, "tflops_tf32_issued": tf32_issued,
+                    "tf32_peak": TF32_OVER_BF16 * tf, "frac_of_tf32_tensor": tf32_issued / (TF32_OVER_BF16 * tf)},
     }
     dominant = max((("pack", t_pack), ("restore", t_restore), ("refresh", t_refresh)), key=lambda x: x[1])[0]
     roofline = dict(rl[dominant])
@@ -388,23 +438,117 @@ def main():
         "metric": "pack_restore_GBps", "value": world * (pack_bytes + restore_bytes) / ((t_pack + t_restore) * 1e-3) / 1e9,
         "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_total,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "layers": L, "heads": H, "d_k": D, "d_v": D, "requests": N_REQ,
-                   "keep_ratio": KEEP, "suffix_tokens": SUFFIX, "refresh_algo": args.algo,
-                   "l2": "inputs larger than L2 (3 GiB of states, 19 GB of token streams per step)",
+        "config": {"workload": workload_name(c), "kind": c["kind"], "layers": L, "v_heads": H_v, "k_heads": H_k, "d_k": D,
+                   "d_v": D, "requests": N_REQ, "keep_ratio": c["keep"], "suffix_tokens": SUFFIX, "refresh_algo": args.algo,
+                   "stream_layers_resident": group,
+                   "l2": "inputs larger than L2 (GiBs of states and token streams per step); no flush needed",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "ms": {"pack": t_pack, "restore": t_restore, "refresh": t_refresh},
         "pack_GBps": world * pack_gbs, "restore_GBps": world * restore_gbs,
         "refresh_tokens_per_s": world * N_REQ * SUFFIX / (t_refresh * 1e-3),
         "refresh_token_heads_per_s": world * token_heads / (t_refresh * 1e-3),
-        "roofline": roofline, "roofline_by_kernel": rl, "clocks": clocks, "gpu_launches": 3 * args.steps,
+        "roofline": roofline, "roofline_by_kernel": rl, "clocks": clocks,
+        "gpu_launches": (2 + n_groups) * args.steps,
     }
     if e2e:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = {k2: v2 for k2, v2 in oracle_leg().items() if k2 != "seconds"}
+        line["cpu_baseline"] = {k2: v2 for k2, v2 in oracle_leg(c).items() if k2 != "seconds"}
     print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
+
+
+def run_mixed_trace(args, c):
+    """Mixed serving trace (single GPU): waves of new checkpoints are packed on one stream while cached
+    checkpoints are restored and refreshed (ragged suffixes, uniform in [1, 1024]) on another.  The slot pool is
+    one contiguous buffer recycled round-robin.  Reports both streams overlapped and run one after the other."""
+    import paper_2608_30386_b200 as dasc
+    from paper_2608_30386_b200 import synth
+
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    pk = peaks()
+    L, H, wave, n_slots = c["L"], c["H_v"], c["n_req"], 1024
+    plan, rates, gen = build_plan(c, local)
+    dense = H * D * D
+    ls, rs = wave * dense, dense
+    slot = int(plan.slot_floats)
+    dgen = synth.generator(c["seed"], dev)
+    pool = torch.empty((n_slots, slot), device=dev)
+    pool.normal_(generator=dgen)                                       # resident checkpoints to hit
+    new_states = synth.states(dgen, (L, wave, dense), dev)
+    active = torch.empty((L, wave, dense), device=dev)
+    ids = torch.arange(wave, dtype=torch.int32, device=dev)
+    n_waves = args.warmup + args.steps
+    cus = [synth.ragged_cu_seqlens(gen, wave, 1, 1024) for _ in range(n_waves)]
+    t_max = max(int(cu[-1]) for cu in cus)
+    group = 6                                                          # layers of token streams resident at once
+    parts = [synth.token_streams(dgen, synth.KDA, 1, t_max, H, H, D, D, rates[l:l + 1], device=dev) for l in range(group)]
+    q, k, v, g, beta = (torch.cat([getattr(p, f) for p in parts]) for f in ("q", "k", "v", "g", "beta"))
+    del parts
+    o = torch.empty((group, t_max, H, D), dtype=torch.bfloat16, device=dev)
+    ws = torch.zeros(256, dtype=torch.uint8, device=dev)
+    s_pack, s_load = torch.cuda.Stream(), torch.cuda.Stream()
+    cu_dev = [cu.to(dev) for cu in cus]
+    new_slots = [((torch.arange(wave) + 512 + w * wave) % 512 + 512).to(torch.int32).to(dev) for w in range(n_waves)]
+    hit_slots = [torch.randperm(512, generator=gen)[:wave].to(torch.int32).to(dev) for _ in range(n_waves)]
+
+    def pack_side(w):
+        dasc.dasc_pack(plan, new_states, ls, rs, ids, pool, new_slots[w], stream=s_pack)
+
+    def load_side(w):
+        T = int(cus[w][-1])
+        # streams are laid out for t_max tokens per layer; the call sees the first T of each layer
+        dasc.dasc_restore(plan, pool, hit_slots[w], active, ls, rs, ids, stream=s_load)
+        for gi in range(L // group):
+            dasc.dasc_refresh(plan, active, ls, rs, ids, q, k, v, g, beta, cu_dev[w], t_max, 1024,
+                              layer_begin=gi * group, layer_end=(gi + 1) * group, o=o, workspace=ws, stream=s_load)
+
+    def run(overlap):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for w in range(args.warmup):
+            pack_side(w)
+            load_side(w)
+        torch.cuda.synchronize()
+        ev0.record(torch.cuda.current_stream())
+        s_pack.wait_event(ev0)
+        s_load.wait_event(ev0)
+        for w in range(args.warmup, n_waves):
+            pack_side(w)
+            if not overlap:
+                s_load.wait_stream(s_pack)
+            load_side(w)
+            if not overlap:
+                s_pack.wait_stream(s_load)
+        torch.cuda.current_stream().wait_stream(s_pack)
+        torch.cuda.current_stream().wait_stream(s_load)
+        ev1.record(torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1) / args.steps
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    t_serial = run(False)
+    t_overlap = run(True)
+    clocks = sampler.stop()
+    assert dasc.dasc_refresh_status(ws) == 0
+    tokens = sum(int(cu[-1]) for cu in cus[args.warmup:]) / args.steps
+    copy_bytes = (2 * wave * slot + wave * (slot + L * dense)) * 4
+    print(json.dumps({
+        "metric": "pack_restore_GBps", "value": copy_bytes / (t_overlap * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_overlap, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_name(c), "wave_requests": wave, "pool_slots": n_slots,
+                   "suffix_tokens": "uniform in [1, 1024]", "streams": 2,
+                   "note": "value counts pack+restore bytes over the whole overlapped step, refresh included"},
+        "ms_per_step_serial": t_serial, "overlap_speedup": t_serial / t_overlap,
+        "refresh_tokens_per_s": tokens / (t_overlap * 1e-3), "tokens_per_step": tokens, "clocks": clocks,
+        "gpu_launches": (2 + L // group) * args.steps * 2,
+    }))
 
 
 if __name__ == "__main__":
