@@ -1,6 +1,7 @@
-// Suffix refresh, chunked form, on the Blackwell tensor cores (tcgen05 + TMEM).
+// Suffix refresh, chunked form, on the Blackwell tensor cores (tcgen05 + TMEM):
+// 32-token chunks, two CTAs resident per SM.
 //
-// Eq. 1 (transposed orientation) over a chunk of C = 64 tokens starting from S_0, with
+// Eq. 1 (transposed orientation) over a chunk of C = 32 tokens starting from S_0, with
 // G_t the running sum of the log-decay inside the chunk and m the chunk midpoint:
 //   Kt_t = k_t * exp(G_t - G_m),  Kh_t = k_t * exp(G_m - G_t),  Qt_t = q_t * exp(G_t - G_m)
 //   S'   = Diag(exp(G_m)) S_0                                   (state decayed to the midpoint)
@@ -10,23 +11,23 @@
 //   S_C  = Diag(exp(G_C - G_m)) (S' + Kh^T U)
 // Referencing the decay to the midpoint keeps every exponent within half a chunk's decay.
 //
-// Mapping.  One CTA per (request, layer, value head): eight compute warps (256 threads) and
-// one warp that only issues tensor-core work.  The state lives in TMEM transposed, S'^T:
-// lane = value column v, column = key channel c, fp32, for the whole suffix.  All five
-// products run as M = 128 tcgen05.mma (kind::tf32, fp32 accumulate) with the value index on
-// the TMEM lanes, so that each accumulator is directly the A operand of the next:
-//   MMA1  [Kt;Qt] Kh^T            -> A (lanes 0-63) and P (lanes 64-127)        smem x smem
+// Mapping.  One CTA per (request, layer, value head): four compute warps and one warp that only
+// issues tensor-core work; 256 TMEM columns and about 108 KB of shared memory per CTA, so two
+// CTAs share an SM and one fills the other's latency gaps (every phase of a chunk depends on the
+// one before it).  The state lives in TMEM transposed, S'^T: lane = value column v, column = key
+// channel c, fp32, for the whole suffix; the tensor core reads it as a tf32 operand directly.
+// All products are M = 128 tcgen05.mma (kind::tf32, fp32 accumulate) with the value index on the
+// TMEM lanes, so that each accumulator is the A operand of the next product:
+//   MMA1  [Kt;Qt] Kh^T            -> A (lanes 0-31) and P (lanes 32-63)         smem x smem
 //   MMA2  S'^T [Kt;Qt]^T          -> R^T | (Qt S')^T                            tmem x smem
-//   MMA3  RHS^T T^T               -> U^T                                         tmem x smem
+//   MMA3  RHS^T T^T               -> U^T      (RHS as a tf32 high/low pair)     tmem x smem
 //   MMA4  (Qt S')^T += U^T P^T    -> O^T                                         tmem x smem
-//   MMA5  S'^T      += U^T Kh     -> state                                       tmem x smem
-// Operands built on the CUDA cores are rounded to tf32 (round-to-nearest) before use; the
-// state master copy stays fp32.  The unit-lower-triangular inverse T = (I + A)^-1 is formed
-// blockwise: 16x16 diagonal blocks by fp32 substitution, off-diagonal blocks by warp-level
+//   MMA5  S'^T      += U^T Kh     -> state    (U as a tf32 high/low pair)       tmem x smem
+// Operands built on the CUDA cores are rounded to tf32 (round-to-nearest).  T = (I + A)^-1 is
+// formed by one warp: 16x16 diagonal blocks by fp32 substitution, the off-diagonal block by
 // mma.sync (tf32) products.  Token inputs of chunk n+1 are fetched with cp.async while chunk n
-// computes: q, k into their own buffer, g into the triangular work matrices once T is out,
-// v into the V tile once the right-hand side is formed.  Kh[t][c] (needed by MMA1 only)
-// shares its storage with the T and P tiles (written after MMA1 has completed).
+// computes.  Kh[t][c] (needed by MMA1 only) shares its storage with the T and P tiles; the raw
+// log-decay tile shares its storage with the V tile.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -37,44 +38,52 @@ namespace {
 
 using namespace tc5;
 
-constexpr int C = 64;        // chunk length
+constexpr int C = 32;        // chunk length
 constexpr int D = 128;       // d_k = d_v
-constexpr int NC = 256;      // compute threads
+constexpr int NC = 128;      // compute threads
 constexpr int NT = NC + 32;  // + the MMA-issuing warp
-constexpr int LDX = 68;      // row pitch (floats) of the fp32 triangular work matrices
+constexpr int LDX = 36;      // row pitch (floats) of the fp32 triangular work matrices
+constexpr uint32_t TMEM_COLS = 256;
 
 // TMEM columns
-constexpr uint32_t COL_S = 0, COL_SOP = 128, COL_RO = 256, COL_AP = 384, COL_U = 448;
+constexpr uint32_t COL_S = 0, COL_AP = 128, COL_RO = 160, COL_U = 224;  // RO: R^T 160-191 | (Qt S')^T 192-223
 
 // shared memory map (bytes)
-constexpr uint32_t OFF_KQ = 0;                        // [4][128 rows][128 B]  rows 0-63 Kt, 64-127 Qt; later the O tile
-constexpr uint32_t OFF_KHT = OFF_KQ + 4 * 128 * 128;  // [2][128 rows][128 B]  Kh^T[c][t]
-constexpr uint32_t OFF_KH = OFF_KHT + 2 * 128 * 128;  // [4][64 rows][128 B]   Kh[t][c], until MMA1 is done; then:
-constexpr uint32_t OFF_TM = OFF_KH;                   // [2][64 rows][128 B]   T[t][i]
-constexpr uint32_t OFF_PM = OFF_TM + 2 * 64 * 128;    // [2][64 rows][128 B]   P[t][i]
-constexpr uint32_t OFF_RAWQ = OFF_KH + 4 * 64 * 128;  // [64][128] bf16 raw q of the next chunk
-constexpr uint32_t OFF_RAWK = OFF_RAWQ + C * D * 2;   // [64][128] bf16 raw k of the next chunk
-constexpr uint32_t OFF_V = OFF_RAWK + C * D * 2;      // [64][128] bf16
-constexpr uint32_t OFF_L = OFF_V + C * D * 2;         // [64][LDX] fp32                  (raw g of the next chunk
-constexpr uint32_t OFF_X = OFF_L + C * LDX * 4;       // [64][LDX] fp32                   spans L and X)
-constexpr uint32_t OFF_FAC = OFF_X + C * LDX * 4;     // [128] fp32 state factor per channel
-constexpr uint32_t OFF_POST = OFF_FAC + D * 4;        // [2][128] fp32 log-factor owed after a chunk, by chunk parity
-constexpr uint32_t OFF_BETA = OFF_POST + 2 * D * 4;   // [2][64] fp32, by chunk parity
-constexpr uint32_t OFF_GSC = OFF_BETA + 2 * C * 4;    // [2][64] fp32 scalar log-decay (GDN), by chunk parity
-constexpr uint32_t OFF_MISC = OFF_GSC + 2 * C * 4;    // barriers, tmem base, abort flag
+constexpr uint32_t OFF_KQ = 0;                         // [4][64 rows][128 B]  rows 0-31 Kt, 32-63 Qt; later the O tile
+constexpr uint32_t OFF_KHT = OFF_KQ + 4 * 64 * 128;    // [1][128 rows][128 B] Kh^T[c][t]
+constexpr uint32_t OFF_KH = OFF_KHT + 128 * 128;       // [4][32 rows][128 B]  Kh[t][c], until MMA1 is done; then:
+constexpr uint32_t OFF_TM = OFF_KH;                    // [1][32 rows][128 B]  T[t][i]
+constexpr uint32_t OFF_PM = OFF_TM + 32 * 128;         // [1][32 rows][128 B]  P[t][i]
+constexpr uint32_t OFF_RAWQ = OFF_KH + 4 * 32 * 128;   // [32][128] bf16 raw q of the next chunk
+constexpr uint32_t OFF_RAWK = OFF_RAWQ + C * D * 2;    // [32][128] bf16 raw k of the next chunk
+constexpr uint32_t OFF_G = OFF_RAWK + C * D * 2;       // [32][128] fp32 raw g (until prep), then
+constexpr uint32_t OFF_V = OFF_G;                      // [32][128] bf16 v (until the right-hand side is formed)
+constexpr uint32_t OFF_L = OFF_G + C * D * 4;          // [32][LDX] fp32
+constexpr uint32_t OFF_X = OFF_L + C * LDX * 4;        // [32][LDX] fp32
+constexpr uint32_t OFF_FAC = OFF_X + C * LDX * 4;      // [128] fp32 state factor per channel
+constexpr uint32_t OFF_POST = OFF_FAC + D * 4;         // [2][128] fp32 log-factor owed after a chunk, by chunk parity
+constexpr uint32_t OFF_BETA = OFF_POST + 2 * D * 4;    // [2][32] fp32, by chunk parity
+constexpr uint32_t OFF_GSC = OFF_BETA + 2 * C * 4;     // [2][32] fp32 scalar log-decay (GDN), by chunk parity
+constexpr uint32_t OFF_MISC = OFF_GSC + 2 * C * 4;     // barriers, tmem base, abort flag
 constexpr uint32_t SMEM_BYTES = OFF_MISC + 128;
-constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;    // slack to align the base to 1024 bytes
-static_assert(2 * C * LDX * 4 >= C * D * 4, "raw g must fit in the L and X matrices");
-static_assert(SMEM_ALLOC <= 227 * 1024, "shared memory budget");
+constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;     // slack to align the base to 1024 bytes
+static_assert(SMEM_ALLOC <= 113 * 1024, "two CTAs per SM");
 
 constexpr uint32_t kMaxPolls = 1u << 22;
 
-// Optional per-phase cycle counters of CTA 0 (development builds only): accumulated by thread 0
-// and written behind the time-out flag in the workspace.
+// The tensor core reads the fp32 state as tf32 by dropping its low 13 mantissa bits, i.e. rounding
+// towards zero: on average the operand is 2^-11 * E[1/m] = 3.52e-4 too small in magnitude (m the
+// significand, log-uniform in [1, 2)).  The rows of Kt and Qt, the only partners of that operand,
+// are scaled up by this factor to cancel the bias; A and P, which also come from those rows, are
+// scaled back down when they are taken out of TMEM.
+constexpr float kTruncComp = 1.000352f;
+constexpr float kInvTruncComp = 1.0f / kTruncComp;
+constexpr float kLog2TruncComp = 5.0774e-4f;  // log2(kTruncComp)
+
 #ifdef DASC_PHASE_TIMING
 #define PT_DECL long long pt_acc[16] = {0}; long long pt_last = clock64();
 #define PT(i) do { long long pt_now = clock64(); pt_acc[i] += pt_now - pt_last; pt_last = pt_now; } while (0)
-#define PT_DUMP do { if (blockIdx.x == 0 && tid == 0) { long long *d = reinterpret_cast<long long *>(static_cast<char *>(a.workspace) + 64); for (int i = 0; i < 16; ++i) d[i] = pt_acc[i]; } } while (0)
+#define PT_DUMP do { if (blockIdx.x == gridDim.x / 2 && tid == 0) { long long *d = reinterpret_cast<long long *>(static_cast<char *>(a.workspace) + 64); for (int i = 0; i < 16; ++i) d[i] = pt_acc[i]; } } while (0)
 #else
 #define PT_DECL
 #define PT(i)
@@ -84,7 +93,7 @@ constexpr uint32_t kMaxPolls = 1u << 22;
 struct Misc {
   // tensor core -> compute warps (one tcgen05.commit each per chunk)
   uint64_t bar_ap, bar_ro, bar_u, bar_o, bar_s;
-  // compute warps -> issuing warp (256 arrivals each per chunk)
+  // compute warps -> issuing warp (128 arrivals each per chunk)
   uint64_t rdy_prep, rdy_state, rdy_rhs, rdy_u;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
@@ -105,8 +114,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// barrier among the 256 compute threads only
-__device__ __forceinline__ void sync_compute() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// barrier among the 128 compute threads only
+__device__ __forceinline__ void sync_compute() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // Bounded wait; after one time-out every later wait of this CTA returns at once.
 __device__ __forceinline__ void wait_bar(uint64_t *bar, uint32_t parity, Misc *misc, uint32_t *err) {
@@ -151,8 +160,11 @@ __device__ __forceinline__ void warp_mm_store(float *Cb, const float (&acc)[2][4
   }
 }
 
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
 template <bool KDA, typename OT>
-__global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs a) {
+__global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs a) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t{1023});
   const uint32_t sbase = smem_u32(smem);
@@ -163,9 +175,6 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
   float *beta_s = reinterpret_cast<float *>(smem + OFF_BETA);
   float *gsc_s = reinterpret_cast<float *>(smem + OFF_GSC);
   const __nv_bfloat16 *Vs = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_V);
-  const __nv_bfloat16 *Qraw = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_RAWQ);
-  const __nv_bfloat16 *Kraw = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_RAWK);
-  const float *Graw = reinterpret_cast<const float *>(smem + OFF_L);
   Misc *misc = reinterpret_cast<Misc *>(smem + OFF_MISC);
   uint32_t *err = static_cast<uint32_t *>(a.workspace);
 
@@ -205,8 +214,8 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
     misc->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 8) {
-    tmem_alloc(&misc->tmem_base, 512);
+  if (warp == 4) {
+    tmem_alloc(&misc->tmem_base, TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -215,14 +224,16 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
   const uint32_t tm = misc->tmem_base;
   const int n_chunks = (n_tok + C - 1) / C;
 
-  constexpr uint32_t ID_M128_N64 = idesc_tf32(128, 64, false, false);
-  constexpr uint32_t ID_M128_N128 = idesc_tf32(128, 128, false, false);
+  constexpr uint32_t ID_N32 = idesc_tf32(128, 32, false, false);
+  constexpr uint32_t ID_N64 = idesc_tf32(128, 64, false, false);
+  constexpr uint32_t ID_N128 = idesc_tf32(128, 128, false, false);
 
-  if (warp == 8) {
+  if (warp == 4) {
     // =========================== tensor-core issue warp ===========================
     for (int ch = 0; ch < n_chunks; ++ch) {
       const uint32_t par = ch & 1;
-      // MMA1: [Kt;Qt] Kh^T
+      // MMA1: [Kt;Qt] Kh^T.  M is padded to 128: rows 64-127 of the A tile are whatever follows it in
+      // shared memory, and land in TMEM lanes 64-127 that nobody reads.
       if (lane == 0) wait_bar(&misc->rdy_prep, par, misc, err);
       __syncwarp();
       if (lane == 0) {
@@ -231,11 +242,11 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
         for (int kb = 0; kb < 4; ++kb)
 #pragma unroll
           for (int j = 0; j < 4; ++j)
-            mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + kb * (128 * 128) + j * 32),
-                   desc_kmajor(sbase + OFF_KH + kb * (64 * 128) + j * 32), ID_M128_N64, (kb | j) != 0);
+            mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + kb * (64 * 128) + j * 32),
+                   desc_kmajor(sbase + OFF_KH + kb * (32 * 128) + j * 32), ID_N32, (kb | j) != 0);
         mma_commit(&misc->bar_ap);
       }
-      // MMA2: S'^T [Kt;Qt]^T
+      // MMA2: S'^T [Kt;Qt]^T, the fp32 state read as a tf32 operand
       if (lane == 0) wait_bar(&misc->rdy_state, par, misc, err);
       __syncwarp();
       if (lane == 0) {
@@ -244,59 +255,47 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
         for (int kb = 0; kb < 4; ++kb)
 #pragma unroll
           for (int j = 0; j < 4; ++j)
-            mma_ts(tm + COL_RO, tm + COL_SOP + kb * 32 + j * 8, desc_kmajor(sbase + OFF_KQ + kb * (128 * 128) + j * 32),
-                   ID_M128_N128, (kb | j) != 0);
+            mma_ts(tm + COL_RO, tm + COL_S + kb * 32 + j * 8, desc_kmajor(sbase + OFF_KQ + kb * (64 * 128) + j * 32),
+                   ID_N64, (kb | j) != 0);
         mma_commit(&misc->bar_ro);
       }
-      // MMA3: U^T = RHS^T T^T
+      // MMA3: U^T = RHS^T T^T; RHS^T is a tf32 pair (high part over R^T, low part in the A|P columns)
       if (lane == 0) wait_bar(&misc->rdy_rhs, par, misc, err);
       __syncwarp();
       if (lane == 0) {
         tc_fence_after_sync();
-        // RHS^T is given as a tf32 pair (high part over R^T, low part in the A|P columns)
 #pragma unroll
         for (int part = 0; part < 2; ++part)
 #pragma unroll
-          for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              mma_ts(tm + COL_U, tm + (part == 0 ? COL_RO : COL_AP) + kb * 32 + j * 8,
-                     desc_kmajor(sbase + OFF_TM + kb * (64 * 128) + j * 32), ID_M128_N64, (part | kb | j) != 0);
+          for (int j = 0; j < 4; ++j)
+            mma_ts(tm + COL_U, tm + (part == 0 ? COL_RO : COL_AP) + j * 8, desc_kmajor(sbase + OFF_TM + j * 32), ID_N32,
+                   (part | j) != 0);
         mma_commit(&misc->bar_u);
       }
-      // MMA4: O^T += U^T P^T;  MMA5: S'^T += U^T Kh
+      // MMA4: O^T += U^T P^T (high part of U);  MMA5: S'^T += U^T Kh (U as a pair: high in place, low over RHS^T)
       if (lane == 0) wait_bar(&misc->rdy_u, par, misc, err);
       __syncwarp();
       if (lane == 0) {
         tc_fence_after_sync();
-        // U^T is given as a tf32 pair (high part in place, low part over the consumed RHS^T columns)
-        // (the outputs take the high part only: their error budget does not need the low part)
         if (go) {
 #pragma unroll
-          for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              mma_ts(tm + COL_RO + 64, tm + COL_U + kb * 32 + j * 8,
-                     desc_kmajor(sbase + OFF_PM + kb * (64 * 128) + j * 32), ID_M128_N64, true);
+          for (int j = 0; j < 4; ++j)
+            mma_ts(tm + COL_RO + 32, tm + COL_U + j * 8, desc_kmajor(sbase + OFF_PM + j * 32), ID_N32, true);
         }
         mma_commit(&misc->bar_o);
 #pragma unroll
         for (int part = 0; part < 2; ++part)
 #pragma unroll
-          for (int kb = 0; kb < 2; ++kb)
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              mma_ts(tm + COL_S, tm + (part == 0 ? COL_U : COL_RO) + kb * 32 + j * 8,
-                     desc_kmajor(sbase + OFF_KHT + kb * (128 * 128) + j * 32), ID_M128_N128, true);
+          for (int j = 0; j < 4; ++j)
+            mma_ts(tm + COL_S, tm + (part == 0 ? COL_U : COL_RO) + j * 8, desc_kmajor(sbase + OFF_KHT + j * 32), ID_N128,
+                   true);
         mma_commit(&misc->bar_s);
       }
       __syncwarp();
     }
   } else {
     // =============================== compute warps ===============================
-    const int quad = warp & 3, colh = warp >> 2;                           // TMEM lane quadrant, column half
-    const uint32_t tlane = tm + (static_cast<uint32_t>(quad * 32) << 16);  // this warp's TMEM lanes
-    const int vrow = quad * 32 + lane;                                     // the TMEM lane this thread owns
+    const uint32_t tlane = tm + (static_cast<uint32_t>(warp * 32) << 16);  // this warp's TMEM lanes; lane index = tid
     constexpr float LOG2E = 1.4426950408889634f;
     PT_DECL
 
@@ -317,7 +316,7 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
         for (int i = tid; i < C * 32; i += NC) {
           const int t = i >> 5, j = i & 31;
           const bool valid = t < ntok;
-          cp_async16_zfill(sbase + OFF_L + t * 512 + j * 16,
+          cp_async16_zfill(sbase + OFF_G + t * 512 + j * 16,
                            reinterpret_cast<const char *>(gg + (t0 + (valid ? t : 0)) * g_stride) + j * 16, valid);
         }
       }
@@ -331,7 +330,7 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
                          reinterpret_cast<const char *>(gv + (t0 + (valid ? t : 0)) * v_stride) + j * 16, valid);
       }
     };
-    // per-token scalars of a chunk (beta, and the scalar log-decay of GDN): threads 0-63 / 64-127
+    // per-token scalars of a chunk (beta, and the scalar log-decay of GDN): threads 0-31 / 32-63
     auto load_scalar = [&](int ch) -> float {
       const int t0 = ch * C, ntok = min(C, n_tok - t0);
       if (tid < C) return tid < ntok ? gb[(t0 + tid) * b_stride] : 0.f;
@@ -346,19 +345,18 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
     if (n_chunks > 0) {
       stage_qk(0);
       stage_g(0);
-      stage_v(0);
       asm volatile("cp.async.commit_group;" ::: "memory");
       store_scalar(0, load_scalar(0));
     }
-    if (tid < D) post_s[tid] = 0.f;  // nothing owed before the first chunk (parity 1 = "chunk -1")
-    if (tid < D) post_s[D + tid] = 0.f;
+    post_s[tid] = 0.f;  // nothing owed before the first chunk
+    post_s[D + tid] = 0.f;
 
     for (int ch = 0; ch < n_chunks; ++ch) {
       const uint32_t par = ch & 1;
       const int t0 = ch * C;
       const int ntok = min(C, n_tok - t0);
       const bool more = ch + 1 < n_chunks;
-      const float* beta_c = beta_s + par * C;
+      const float *beta_c = beta_s + par * C;
 
       // ---- (1) this chunk's inputs have landed; the previous chunk's state update is complete ----
       if (ch > 0) wait_bar(&misc->bar_s, par ^ 1, misc, err);
@@ -368,56 +366,96 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
       const float scalar_next = more ? load_scalar(ch + 1) : 0.f;  // in flight during the chunk
       PT(0);
 
-      // ---- (2) prep: thread = (key channel c, token half) ----
+      // ---- (2) prep: warp = block of 32 channels; lane = (4 adjacent channels, 8 consecutive tokens) ----
       {
-        const int c = tid & (D - 1), half = tid >> 7;
-        const int tb = half * (C / 2);
-        float G[C / 2];
+        const int cq = lane & 7, tg = lane >> 3;
+        const int c0 = warp * 32 + cq * 4, tb = tg * 8;
+        float G[8][4];
 #pragma unroll
-        for (int t = 0; t < C / 2; ++t) G[t] = KDA ? Graw[(tb + t) * D + c] : gsc_s[par * C + tb + t];
-#pragma unroll
-        for (int t = 1; t < C / 2; ++t) G[t] += G[t - 1];
-        // the midpoint is the end of the first half: first-half exponents are G_t - G_m = G[t] - G[31],
-        // second-half exponents are the local running sums themselves
-        const float ref = half == 0 ? G[C / 2 - 1] : 0.f;
-        if (half == 0) fac_s[c] = ex2f((post_s[(par ^ 1) * D + c] + G[C / 2 - 1]) * LOG2E);
-        else post_s[par * D + c] = G[C / 2 - 1];  // G_C - G_m, owed to the state after this chunk
-#pragma unroll
-        for (int t4 = 0; t4 < C / 2; t4 += 4) {
-          uint32_t kht[4];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int t = tb + t4 + u;
-            const float kf = __bfloat162float(Kraw[t * D + c]);
-            const float qf = __bfloat162float(Qraw[t * D + c]) * a.q_scale;
-            const float d = (G[t4 + u] - ref) * LOG2E;
-            const float e1 = ex2f(d), e2 = ex2f(-d);
-            *reinterpret_cast<uint32_t *>(smem + OFF_KQ + sw128_offset(128, t, c)) = to_tf32(kf * e1);
-            *reinterpret_cast<uint32_t *>(smem + OFF_KQ + sw128_offset(128, 64 + t, c)) = to_tf32(qf * e1);
-            kht[u] = to_tf32(kf * e2);
-            *reinterpret_cast<uint32_t *>(smem + OFF_KH + sw128_offset(64, t, c)) = kht[u];
+        for (int j = 0; j < 8; ++j) {
+          if constexpr (KDA) {
+            const float4 gv4 = *reinterpret_cast<const float4 *>(smem + OFF_G + (tb + j) * 512 + c0 * 4);
+            G[j][0] = gv4.x; G[j][1] = gv4.y; G[j][2] = gv4.z; G[j][3] = gv4.w;
+          } else {
+            const float gs = gsc_s[par * C + tb + j];
+            G[j][0] = gs; G[j][1] = gs; G[j][2] = gs; G[j][3] = gs;
           }
-          *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c, tb + t4)) = make_uint4(kht[0], kht[1], kht[2], kht[3]);
+        }
+#pragma unroll
+        for (int j = 1; j < 8; ++j)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) G[j][i] += G[j - 1][i];
+        // prefix over the four token groups of the warp (lanes 8 apart), then the two reference points
+        float Gm[4], Gc[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float incl = G[7][i];
+          const float own = incl;
+          float x = __shfl_up_sync(0xffffffffu, incl, 8);
+          if (tg >= 1) incl += x;
+          x = __shfl_up_sync(0xffffffffu, incl, 16);
+          if (tg >= 2) incl += x;
+          const float off = incl - own;
+          Gm[i] = __shfl_sync(0xffffffffu, incl, cq + 8);   // through token 15: the chunk midpoint
+          Gc[i] = __shfl_sync(0xffffffffu, incl, cq + 24);  // through token 31
+#pragma unroll
+          for (int j = 0; j < 8; ++j) G[j][i] += off;
+        }
+        if (tg == 0) {
+          const float4 pp = *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0);
+          *reinterpret_cast<float4 *>(fac_s + c0) = make_float4(ex2f((pp.x + Gm[0]) * LOG2E), ex2f((pp.y + Gm[1]) * LOG2E),
+                                                                ex2f((pp.z + Gm[2]) * LOG2E), ex2f((pp.w + Gm[3]) * LOG2E));
+        } else if (tg == 1) {
+          *reinterpret_cast<float4 *>(post_s + par * D + c0) = make_float4(Gc[0] - Gm[0], Gc[1] - Gm[1], Gc[2] - Gm[2], Gc[3] - Gm[3]);
+        }
+        uint32_t kht[4][8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int t = tb + j;
+          const uint2 kw = *reinterpret_cast<const uint2 *>(smem + OFF_RAWK + t * 256 + c0 * 2);
+          const uint2 qw = *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + t * 256 + c0 * 2);
+          const float kf[4] = {bf16lo(kw.x), bf16hi(kw.x), bf16lo(kw.y), bf16hi(kw.y)};
+          const float qf[4] = {bf16lo(qw.x), bf16hi(qw.x), bf16lo(qw.y), bf16hi(qw.y)};
+          uint32_t kt[4], qt[4], kh[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float d = (G[j][i] - Gm[i]) * LOG2E;
+            const float e1 = ex2f(d + kLog2TruncComp), e2 = ex2f(-d);
+            kt[i] = to_tf32(kf[i] * e1);
+            qt[i] = to_tf32(qf[i] * a.q_scale * e1);
+            kh[i] = to_tf32(kf[i] * e2);
+            kht[i][j] = kh[i];
+          }
+          *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, t, c0)) = make_uint4(kt[0], kt[1], kt[2], kt[3]);
+          *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, 32 + t, c0)) = make_uint4(qt[0], qt[1], qt[2], qt[3]);
+          *reinterpret_cast<uint4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_uint4(kh[0], kh[1], kh[2], kh[3]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c0 + i, tb)) =
+              make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
+          *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c0 + i, tb + 4)) =
+              make_uint4(kht[i][4], kht[i][5], kht[i][6], kht[i][7]);
         }
       }
       fence_smem_to_async();
       tc_fence_before_sync();
       mbar_arrive(&misc->rdy_prep);  // -> MMA1
       sync_compute();                // fac_s visible; raw q/k/g consumed by everyone
+      stage_v(ch);                   // V of this chunk takes the place of the raw log-decay tile
+      asm volatile("cp.async.commit_group;" ::: "memory");
       if (more) stage_qk(ch + 1);
       asm volatile("cp.async.commit_group;" ::: "memory");
       PT(1);
 
-      // ---- (3) state pass: thread = (value column v, half of the channels); scale to this chunk's
-      //          midpoint and refresh the tf32 operand copy ----
+      // ---- (3) state pass: thread = value column v; scale the state to this chunk's midpoint ----
       {
-        const int cb = colh * 64;
         uint32_t s[2][32];
         auto fetch = [&](int c0, uint32_t(&dst)[32]) {
           if (ch == 0) {
             if (a.mode == DASC_REFRESH_CONTINUE) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) dst[j] = __float_as_uint(st[(c0 + j) * D + vrow]);
+              for (int j = 0; j < 32; ++j) dst[j] = __float_as_uint(st[(c0 + j) * D + tid]);
             } else {
 #pragma unroll
               for (int j = 0; j < 32; ++j) dst[j] = 0u;
@@ -426,25 +464,22 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
             tmem_ld32(tlane + COL_S + c0, dst);
           }
         };
-        fetch(cb, s[0]);
+        fetch(0, s[0]);
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const int c0 = cb + i * 32;
+        for (int i = 0; i < 4; ++i) {
+          const int c0 = i * 32;
           if (ch != 0) tmem_ld_wait();
-          if (i < 1) fetch(c0 + 32, s[(i + 1) & 1]);
+          if (i < 3) fetch(c0 + 32, s[(i + 1) & 1]);
           uint32_t(&cur)[32] = s[i & 1];
-          uint32_t sop[32];
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             const float4 f = *reinterpret_cast<const float4 *>(fac_s + c0 + j);
-            const float x0 = __uint_as_float(cur[j + 0]) * f.x, x1 = __uint_as_float(cur[j + 1]) * f.y;
-            const float x2 = __uint_as_float(cur[j + 2]) * f.z, x3 = __uint_as_float(cur[j + 3]) * f.w;
-            cur[j + 0] = __float_as_uint(x0); cur[j + 1] = __float_as_uint(x1);
-            cur[j + 2] = __float_as_uint(x2); cur[j + 3] = __float_as_uint(x3);
-            sop[j + 0] = to_tf32(x0); sop[j + 1] = to_tf32(x1); sop[j + 2] = to_tf32(x2); sop[j + 3] = to_tf32(x3);
+            cur[j + 0] = __float_as_uint(__uint_as_float(cur[j + 0]) * f.x);
+            cur[j + 1] = __float_as_uint(__uint_as_float(cur[j + 1]) * f.y);
+            cur[j + 2] = __float_as_uint(__uint_as_float(cur[j + 2]) * f.z);
+            cur[j + 3] = __float_as_uint(__uint_as_float(cur[j + 3]) * f.w);
           }
           tmem_st32(tlane + COL_S + c0, cur);
-          tmem_st32(tlane + COL_SOP + c0, sop);
         }
         tmem_st_wait();
       }
@@ -452,172 +487,125 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
       mbar_arrive(&misc->rdy_state);  // -> MMA2
       PT(2);
 
-      // ---- (4) A and P out of TMEM; T = (I + A)^-1 ----
+      // ---- (4) A and P out of TMEM; T = (I + A)^-1, by warp 0 (A) and warp 1 (P) ----
       wait_bar(&misc->bar_ap, par, misc, err);
       tc_fence_after_sync();
       PT(3);
-      {
+      if (warp < 2) {
         uint32_t x[32];
-        const int ib = colh * 32;  // this thread's 32 columns of row `vrow`
-        tmem_ld32(tlane + COL_AP + ib, x);
+        tmem_ld32(tlane + COL_AP, x);
         tmem_ld_wait();
-        if (vrow < C) {
-          // lanes 0-63: row t of A = strict_lower(Kt Kh^T) * beta_t, kept in fp32 for the inverse
-          const int t = vrow;
-          const float bt = beta_c[t];
+        const int t = lane;
+        if (warp == 0) {
+          // lanes 0-31: row t of A = strict_lower(Kt Kh^T) * beta_t, kept in fp32 for the inverse
+          const float bt = beta_c[t] * kInvTruncComp;
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
-            const int i0 = ib + j;
             float4 o;
-            o.x = (i0 + 0 < t) ? bt * __uint_as_float(x[j + 0]) : 0.f;
-            o.y = (i0 + 1 < t) ? bt * __uint_as_float(x[j + 1]) : 0.f;
-            o.z = (i0 + 2 < t) ? bt * __uint_as_float(x[j + 2]) : 0.f;
-            o.w = (i0 + 3 < t) ? bt * __uint_as_float(x[j + 3]) : 0.f;
-            *reinterpret_cast<float4 *>(Lm + t * LDX + i0) = o;
+            o.x = (j + 0 < t) ? bt * __uint_as_float(x[j + 0]) : 0.f;
+            o.y = (j + 1 < t) ? bt * __uint_as_float(x[j + 1]) : 0.f;
+            o.z = (j + 2 < t) ? bt * __uint_as_float(x[j + 2]) : 0.f;
+            o.w = (j + 3 < t) ? bt * __uint_as_float(x[j + 3]) : 0.f;
+            *reinterpret_cast<float4 *>(Lm + t * LDX + j) = o;
+          }
+          __syncwarp();
+          // diagonal 16x16 blocks: lane (block b, column cc) solves (I + L_bb) x = e_cc by forward substitution
+          {
+            const int b = lane >> 4, cc = lane & 15;
+            const float *Lb = Lm + (b * 16) * LDX + b * 16;
+            float xs[16];
+#pragma unroll
+            for (int rr = 0; rr < 16; ++rr) {
+              float acc0 = (rr == cc) ? 1.f : 0.f, acc1 = 0.f;
+#pragma unroll
+              for (int j = 0; j + 1 < rr; j += 2) {
+                acc0 = fmaf(-Lb[rr * LDX + j], xs[j], acc0);
+                acc1 = fmaf(-Lb[rr * LDX + j + 1], xs[j + 1], acc1);
+              }
+              if (rr & 1) acc0 = fmaf(-Lb[rr * LDX + rr - 1], xs[rr - 1], acc0);
+              xs[rr] = acc0 + acc1;
+            }
+#pragma unroll
+            for (int rr = 0; rr < 16; ++rr) Xm[(b * 16 + rr) * LDX + b * 16 + cc] = xs[rr];
+          }
+          __syncwarp();
+          // off-diagonal block: X_10 = -X_11 (L_10 X_00); the product L_10 X_00 is parked in the unused block (0,1)
+          {
+            float acc[2][4] = {};
+            warp_mm_acc(acc, Lm + 16 * LDX, Xm, lane);
+            warp_mm_store(Xm + 16, acc, 1.f, lane);
+            __syncwarp();
+            float acc2[2][4] = {};
+            warp_mm_acc(acc2, Xm + 16 * LDX + 16, Xm + 16, lane);
+            warp_mm_store(Xm + 16 * LDX, acc2, -1.f, lane);
           }
         } else {
-          // lanes 64-127: row t of P = lower_incl_diag(Qt Kh^T), straight to its operand tile
-          const int t = vrow - C;
+          // lanes 32-63: row t of P = lower_incl_diag(Qt Kh^T), straight to its operand tile
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
-            const int i0 = ib + j;
             uint4 o;
-            o.x = (i0 + 0 <= t) ? to_tf32(__uint_as_float(x[j + 0])) : 0u;
-            o.y = (i0 + 1 <= t) ? to_tf32(__uint_as_float(x[j + 1])) : 0u;
-            o.z = (i0 + 2 <= t) ? to_tf32(__uint_as_float(x[j + 2])) : 0u;
-            o.w = (i0 + 3 <= t) ? to_tf32(__uint_as_float(x[j + 3])) : 0u;
-            *reinterpret_cast<uint4 *>(smem + OFF_PM + sw128_offset(64, t, i0)) = o;
+            o.x = (j + 0 <= t) ? to_tf32(__uint_as_float(x[j + 0]) * kInvTruncComp) : 0u;
+            o.y = (j + 1 <= t) ? to_tf32(__uint_as_float(x[j + 1]) * kInvTruncComp) : 0u;
+            o.z = (j + 2 <= t) ? to_tf32(__uint_as_float(x[j + 2]) * kInvTruncComp) : 0u;
+            o.w = (j + 3 <= t) ? to_tf32(__uint_as_float(x[j + 3]) * kInvTruncComp) : 0u;
+            *reinterpret_cast<uint4 *>(smem + OFF_PM + sw128_offset(32, t, j)) = o;
           }
         }
       }
       sync_compute();
       PT(4);
-      // diagonal 16x16 blocks: thread (block b, column cc) solves (I + L_bb) x = e_cc by forward substitution
-      if (tid < C) {
-        const int b = tid >> 4, cc = tid & 15;
-        const float *Lb = Lm + (b * 16) * LDX + b * 16;
-        float x[16];
-#pragma unroll
-        for (int rr = 0; rr < 16; ++rr) {
-          float acc0 = (rr == cc) ? 1.f : 0.f, acc1 = 0.f;
-#pragma unroll
-          for (int j = 0; j + 1 < rr; j += 2) {
-            acc0 = fmaf(-Lb[rr * LDX + j], x[j], acc0);
-            acc1 = fmaf(-Lb[rr * LDX + j + 1], x[j + 1], acc1);
-          }
-          if (rr & 1) acc0 = fmaf(-Lb[rr * LDX + rr - 1], x[rr - 1], acc0);
-          x[rr] = acc0 + acc1;
-        }
-#pragma unroll
-        for (int rr = 0; rr < 16; ++rr) Xm[(b * 16 + rr) * LDX + b * 16 + cc] = x[rr];
-      }
-      sync_compute();
-      PT(5);
       {
-        // off-diagonal blocks, X_IJ = -X_II sum_K L_IK X_KJ; Y_IJ = sum_K L_IK X_KJ is parked in the
-        // (otherwise unused) upper block (J, I) of X.  One warp per block product.
-        auto Lb = [&](int I, int J) { return Lm + (I * 16) * LDX + J * 16; };
-        auto Xb = [&](int I, int J) { return Xm + (I * 16) * LDX + J * 16; };
-        float acc[2][4];
-        auto zero = [&]() {
+        // T (lower triangle of X, unit diagonal) -> tf32 operand tile; 8 elements per thread
+        const int t = tid >> 2, i0 = (tid & 3) * 8;
 #pragma unroll
-          for (int i = 0; i < 2; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-        };
-        // first sub-diagonal: (1,0), (2,1), (3,2)
-        if (warp < 3) {
-          const int I = warp + 1, J = warp;
-          zero();
-          warp_mm_acc(acc, Lb(I, J), Xb(J, J), lane);
-          warp_mm_store(Xb(J, I), acc, 1.f, lane);
-          __syncwarp();
-          zero();
-          warp_mm_acc(acc, Xb(I, I), Xb(J, I), lane);
-          warp_mm_store(Xb(I, J), acc, -1.f, lane);
-        }
-        sync_compute();
-        // second sub-diagonal: (2,0), (3,1)
-        if (warp < 2) {
-          const int I = warp + 2, J = warp;
-          zero();
-          warp_mm_acc(acc, Lb(I, J), Xb(J, J), lane);
-          warp_mm_acc(acc, Lb(I, J + 1), Xb(J + 1, J), lane);
-          warp_mm_store(Xb(J, I), acc, 1.f, lane);
-          __syncwarp();
-          zero();
-          warp_mm_acc(acc, Xb(I, I), Xb(J, I), lane);
-          warp_mm_store(Xb(I, J), acc, -1.f, lane);
-        }
-        sync_compute();
-        // corner block (3,0)
-        if (warp == 0) {
-          zero();
-          warp_mm_acc(acc, Lb(3, 0), Xb(0, 0), lane);
-          warp_mm_acc(acc, Lb(3, 1), Xb(1, 0), lane);
-          warp_mm_acc(acc, Lb(3, 2), Xb(2, 0), lane);
-          warp_mm_store(Xb(0, 3), acc, 1.f, lane);
-          __syncwarp();
-          zero();
-          warp_mm_acc(acc, Xb(3, 3), Xb(0, 3), lane);
-          warp_mm_store(Xb(3, 0), acc, -1.f, lane);
-        }
-        sync_compute();
-        // T (lower triangle of X, unit diagonal) -> tf32 operand tile
-        const int t = tid >> 2, i0 = (tid & 3) * 16;
-#pragma unroll
-        for (int j = 0; j < 16; j += 4) {
+        for (int j = 0; j < 8; j += 4) {
           const float4 xv = *reinterpret_cast<const float4 *>(Xm + t * LDX + i0 + j);
           uint4 o;
           o.x = (i0 + j + 0 <= t) ? to_tf32(xv.x) : 0u;
           o.y = (i0 + j + 1 <= t) ? to_tf32(xv.y) : 0u;
           o.z = (i0 + j + 2 <= t) ? to_tf32(xv.z) : 0u;
           o.w = (i0 + j + 3 <= t) ? to_tf32(xv.w) : 0u;
-          *reinterpret_cast<uint4 *>(smem + OFF_TM + sw128_offset(64, t, i0 + j)) = o;
+          *reinterpret_cast<uint4 *>(smem + OFF_TM + sw128_offset(32, t, i0 + j)) = o;
         }
       }
       fence_smem_to_async();
-      sync_compute();  // everyone is done with L and X: the next chunk's g may land there
-      if (more) stage_g(ch + 1);
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      PT(6);
+      PT(5);
 
-      // ---- (5) RHS^T = beta (V - R)^T, written over R^T as the tf32 A operand of MMA3 ----
+      // ---- (5) RHS^T = beta (V - R)^T as a tf32 pair: high over R^T, low in the consumed A|P columns ----
       wait_bar(&misc->bar_ro, par, misc, err);
       tc_fence_after_sync();
-      PT(7);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");  // V of this chunk (the newer group is the next q, k)
+      sync_compute();
+      PT(6);
       {
-        const int tb = colh * 32;
         uint32_t x[32], lo[32];
-        tmem_ld32(tlane + COL_RO + tb, x);
+        tmem_ld32(tlane + COL_RO, x);
         tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-          const int t = tb + j;
-          const float vv = __bfloat162float(Vs[t * D + vrow]);
-          const float rhs = beta_c[t] * (vv - __uint_as_float(x[j]));
-          x[j] = to_tf32(rhs);                                  // high part
-          lo[j] = to_tf32(rhs - __uint_as_float(x[j]));         // what the high part lost
+          const float vv = __bfloat162float(Vs[j * D + tid]);
+          const float rhs = beta_c[j] * (vv - __uint_as_float(x[j]));
+          x[j] = to_tf32(rhs);
+          lo[j] = to_tf32(rhs - __uint_as_float(x[j]));
         }
-        tmem_st32(tlane + COL_RO + tb, x);
-        tmem_st32(tlane + COL_AP + tb, lo);  // the A|P columns were consumed in step (4)
+        tmem_st32(tlane + COL_RO, x);
+        tmem_st32(tlane + COL_AP, lo);
         tmem_st_wait();
       }
       tc_fence_before_sync();
       mbar_arrive(&misc->rdy_rhs);  // -> MMA3 (T tile and RHS^T are ready)
-      sync_compute();               // everyone is done with V: the next chunk's tile may land
-      if (more) stage_v(ch + 1);
+      sync_compute();               // everyone is done with V: the next chunk's log-decay tile may land
+      if (more) stage_g(ch + 1);
       asm volatile("cp.async.commit_group;" ::: "memory");
-      PT(8);
+      PT(7);
 
-      // ---- (6) U^T rounded to tf32 in place ----
+      // ---- (6) U^T as a tf32 pair: high in place, low over the consumed RHS^T ----
       wait_bar(&misc->bar_u, par, misc, err);
       tc_fence_after_sync();
-      PT(9);
+      PT(8);
       {
-        const int tb = colh * 32;
         uint32_t x[32], lo[32];
-        tmem_ld32(tlane + COL_U + tb, x);
+        tmem_ld32(tlane + COL_U, x);
         tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
@@ -625,28 +613,27 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
           x[j] = to_tf32(u);
           lo[j] = to_tf32(u - __uint_as_float(x[j]));
         }
-        tmem_st32(tlane + COL_U + tb, x);
-        tmem_st32(tlane + COL_RO + tb, lo);  // RHS^T has been consumed by MMA3
+        tmem_st32(tlane + COL_U, x);
+        tmem_st32(tlane + COL_RO, lo);
         tmem_st_wait();
       }
       tc_fence_before_sync();
       mbar_arrive(&misc->rdy_u);  // -> MMA4, MMA5
-      PT(10);
+      PT(9);
 
       // ---- (7) outputs of this chunk ----
       wait_bar(&misc->bar_o, par, misc, err);
       tc_fence_after_sync();
-      PT(11);
+      PT(10);
       if (go) {
-        const int tb = colh * 32;
         uint32_t x[32];
-        tmem_ld32(tlane + COL_RO + 64 + tb, x);
+        tmem_ld32(tlane + COL_RO + 32, x);
         tmem_ld_wait();
         if constexpr (sizeof(OT) == 2) {
           // through shared memory (the Kt/Qt tile is free now) so that global stores are 16 bytes wide
           __nv_bfloat16 *Os = reinterpret_cast<__nv_bfloat16 *>(smem + OFF_KQ);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) Os[(tb + j) * D + vrow] = __float2bfloat16_rn(__uint_as_float(x[j]));
+          for (int j = 0; j < 32; ++j) Os[j * D + tid] = __float2bfloat16_rn(__uint_as_float(x[j]));
           sync_compute();
           for (int i = tid; i < ntok * 16; i += NC) {
             const int t = i >> 4, j = i & 15;
@@ -656,25 +643,25 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (tb + j < ntok) go[(t0 + tb + j) * v_stride + vrow] = __uint_as_float(x[j]);
+            if (j < ntok) go[(t0 + j) * v_stride + tid] = __uint_as_float(x[j]);
         }
       }
       store_scalar(ch + 1, scalar_next);
       tc_fence_before_sync();
       sync_compute();  // every thread is done with this chunk's tiles before they are rewritten
-      PT(12);
+      PT(11);
     }
 
     // ---- final state: the factor still owed, then write back ----
     if (n_chunks > 0) wait_bar(&misc->bar_s, (n_chunks - 1) & 1, misc, err);
-    if (tid < D) fac_s[tid] = ex2f(post_s[((n_chunks + 1) & 1) * D + tid] * LOG2E);
+    fac_s[tid] = ex2f(post_s[((n_chunks + 1) & 1) * D + tid] * LOG2E);
     sync_compute();
     tc_fence_after_sync();
     {
       const uint8_t *keep = a.row_keep + static_cast<int64_t>(layer) * a.rows_per_layer + static_cast<int64_t>(h) * D;
       const bool merge = a.mode != DASC_REFRESH_CONTINUE;
 #pragma unroll 1
-      for (int c0 = colh * 64; c0 < colh * 64 + 64; c0 += 32) {
+      for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t s[32];
         if (n_chunks > 0) {
           tmem_ld32(tlane + COL_S + c0, s);
@@ -686,16 +673,16 @@ __global__ void __launch_bounds__(NT, 1) refresh_chunked_kernel(DascRefreshArgs 
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const int c = c0 + j;
-          if (!merge || !keep[c]) st[c * D + vrow] = __uint_as_float(s[j]) * fac_s[c];
+          if (!merge || !keep[c]) st[c * D + tid] = __uint_as_float(s[j]) * fac_s[c];
         }
       }
     }
-    PT(13);
+    PT(12);
     PT_DUMP;
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 8) tmem_dealloc(tm, 512);
+  if (warp == 4) tmem_dealloc(tm, TMEM_COLS);
 }
 
 template <bool KDA, typename OT>
