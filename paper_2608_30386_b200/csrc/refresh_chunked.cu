@@ -138,15 +138,15 @@ __device__ __forceinline__ void warp_mm_acc(float (&acc)[2][4], const float *A, 
 #pragma unroll
   for (int kh = 0; kh < 2; ++kh) {
     uint32_t af[4];
-    af[0] = to_tf32(A[g * LDX + 8 * kh + tig]);
-    af[1] = to_tf32(A[(g + 8) * LDX + 8 * kh + tig]);
-    af[2] = to_tf32(A[g * LDX + 8 * kh + tig + 4]);
-    af[3] = to_tf32(A[(g + 8) * LDX + 8 * kh + tig + 4]);
+    af[0] = tf32_pre(A[g * LDX + 8 * kh + tig]);
+    af[1] = tf32_pre(A[(g + 8) * LDX + 8 * kh + tig]);
+    af[2] = tf32_pre(A[g * LDX + 8 * kh + tig + 4]);
+    af[3] = tf32_pre(A[(g + 8) * LDX + 8 * kh + tig + 4]);
 #pragma unroll
     for (int nh = 0; nh < 2; ++nh) {
       uint32_t bf[2];
-      bf[0] = to_tf32(B[(8 * kh + tig) * LDX + 8 * nh + g]);
-      bf[1] = to_tf32(B[(8 * kh + tig + 4) * LDX + 8 * nh + g]);
+      bf[0] = tf32_pre(B[(8 * kh + tig) * LDX + 8 * nh + g]);
+      bf[1] = tf32_pre(B[(8 * kh + tig + 4) * LDX + 8 * nh + g]);
       mma_tf32_16x8x8(acc[nh], af, bf);
     }
   }
@@ -421,9 +421,9 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           for (int i = 0; i < 4; ++i) {
             const float d = (G[j][i] - Gm[i]) * LOG2E;
             const float e1 = ex2f(d + kLog2TruncComp), e2 = ex2f(-d);
-            kt[i] = to_tf32(kf[i] * e1);
-            qt[i] = to_tf32(qf[i] * a.q_scale * e1);
-            kh[i] = to_tf32(kf[i] * e2);
+            kt[i] = tf32_pre(kf[i] * e1);
+            qt[i] = tf32_pre(qf[i] * a.q_scale * e1);
+            kh[i] = tf32_pre(kf[i] * e2);
             kht[i][j] = kh[i];
           }
           *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, t, c0)) = make_uint4(kt[0], kt[1], kt[2], kt[3]);
@@ -544,10 +544,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             uint4 o;
-            o.x = (j + 0 <= t) ? to_tf32(__uint_as_float(x[j + 0]) * kInvTruncComp) : 0u;
-            o.y = (j + 1 <= t) ? to_tf32(__uint_as_float(x[j + 1]) * kInvTruncComp) : 0u;
-            o.z = (j + 2 <= t) ? to_tf32(__uint_as_float(x[j + 2]) * kInvTruncComp) : 0u;
-            o.w = (j + 3 <= t) ? to_tf32(__uint_as_float(x[j + 3]) * kInvTruncComp) : 0u;
+            o.x = (j + 0 <= t) ? tf32_pre(__uint_as_float(x[j + 0]) * kInvTruncComp) : 0u;
+            o.y = (j + 1 <= t) ? tf32_pre(__uint_as_float(x[j + 1]) * kInvTruncComp) : 0u;
+            o.z = (j + 2 <= t) ? tf32_pre(__uint_as_float(x[j + 2]) * kInvTruncComp) : 0u;
+            o.w = (j + 3 <= t) ? tf32_pre(__uint_as_float(x[j + 3]) * kInvTruncComp) : 0u;
             *reinterpret_cast<uint4 *>(smem + OFF_PM + sw128_offset(32, t, j)) = o;
           }
         }
@@ -561,10 +561,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         for (int j = 0; j < 8; j += 4) {
           const float4 xv = *reinterpret_cast<const float4 *>(Xm + t * LDX + i0 + j);
           uint4 o;
-          o.x = (i0 + j + 0 <= t) ? to_tf32(xv.x) : 0u;
-          o.y = (i0 + j + 1 <= t) ? to_tf32(xv.y) : 0u;
-          o.z = (i0 + j + 2 <= t) ? to_tf32(xv.z) : 0u;
-          o.w = (i0 + j + 3 <= t) ? to_tf32(xv.w) : 0u;
+          o.x = (i0 + j + 0 <= t) ? tf32_pre(xv.x) : 0u;
+          o.y = (i0 + j + 1 <= t) ? tf32_pre(xv.y) : 0u;
+          o.z = (i0 + j + 2 <= t) ? tf32_pre(xv.z) : 0u;
+          o.w = (i0 + j + 3 <= t) ? tf32_pre(xv.w) : 0u;
           *reinterpret_cast<uint4 *>(smem + OFF_TM + sw128_offset(32, t, i0 + j)) = o;
         }
       }
@@ -586,7 +586,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           const float vv = __bfloat162float(Vs[j * D + tid]);
           const float rhs = beta_c[j] * (vv - __uint_as_float(x[j]));
           x[j] = to_tf32(rhs);
-          lo[j] = to_tf32(rhs - __uint_as_float(x[j]));
+          lo[j] = tf32_pre(rhs - __uint_as_float(x[j]));
         }
         tmem_st32(tlane + COL_RO, x);
         tmem_st32(tlane + COL_AP, lo);
@@ -611,7 +611,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         for (int j = 0; j < 32; ++j) {
           const float u = __uint_as_float(x[j]);
           x[j] = to_tf32(u);
-          lo[j] = to_tf32(u - __uint_as_float(x[j]));
+          lo[j] = tf32_pre(u - __uint_as_float(x[j]));
         }
         tmem_st32(tlane + COL_U, x);
         tmem_st32(tlane + COL_RO, lo);

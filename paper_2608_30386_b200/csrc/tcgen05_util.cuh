@@ -68,6 +68,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
+// 32 lanes x 16 consecutive columns.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -84,18 +100,21 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // ---- operands -------------------------------------------------------------------------------
-// fp32 -> tf32, round to nearest (ties away); the result keeps the fp32 container.
-__device__ __forceinline__ uint32_t to_tf32(float x) {
-  uint32_t r;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-  return r;
-}
+// fp32 -> tf32.  The tensor cores read a tf32 operand from an fp32 container by ignoring the low
+// 13 mantissa bits, so adding half a tf32 ulp to the bit pattern beforehand turns that truncation
+// into round-to-nearest (ties away).  Plain integer arithmetic: cvt.rna.tf32.f32 was measured to
+// cost an order of magnitude more issue time on this part.
+// tf32_pre(x): container whose truncation is the rounded value (for operands only tensor cores read).
+__device__ __forceinline__ uint32_t tf32_pre(float x) { return __float_as_uint(x) + 0x1000u; }
+// to_tf32(x): the rounded value itself, low 13 bits cleared.
+__device__ __forceinline__ uint32_t to_tf32(float x) { return (__float_as_uint(x) + 0x1000u) & 0xFFFFE000u; }
 
 // Shared-memory operand tiles use the 128-byte-swizzle canonical layout.  A tile of R rows
 // and 32*NB tf32 columns is stored as NB blocks of [R rows][128 bytes]; inside a block the
 // 16-byte chunk j of row r sits at chunk position j ^ (r & 7).  Blocks start 1024-byte aligned.
-// The same bytes serve as a K-major operand (rows = M or N index, columns = K) and as an
-// MN-major operand (rows = K index, columns = M or N), only the descriptor differs.
+// These tiles are used as K-major operands (rows = M or N index, columns = K).  A tf32 MN-major
+// operand would need a different swizzle (128-byte swizzle on 32-byte units), so a matrix that is
+// consumed in both orientations is stored twice.
 __device__ __forceinline__ uint32_t sw128_offset(uint32_t rows, uint32_t r, uint32_t col) {
   const uint32_t blk = col >> 5, cin = col & 31;
   return blk * rows * 128u + r * 128u + ((((cin >> 2) ^ (r & 7u)) << 4) | ((cin & 3u) << 2));
@@ -107,13 +126,6 @@ constexpr uint64_t kDescSw128 = (uint64_t{1} << 46) | (uint64_t{2} << 61);  // v
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t smem_addr) {
   return kDescSw128 | (uint64_t{(smem_addr & 0x3FFFFu) >> 4}) | (uint64_t{1} << 16) | (uint64_t{1024 >> 4} << 32);
 }
-// MN-major: the next 32 columns (128 bytes) of the MN extent are `block_bytes` away (LBO);
-// the next 8 K rows are 1024 bytes away (SBO).
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t smem_addr, uint32_t block_bytes) {
-  return kDescSw128 | (uint64_t{(smem_addr & 0x3FFFFu) >> 4}) | (uint64_t{(block_bytes >> 4) & 0x3FFFu} << 16) |
-         (uint64_t{1024 >> 4} << 32);
-}
-
 // Instruction descriptor, kind::tf32, fp32 accumulation.
 __host__ __device__ constexpr uint32_t idesc_tf32(uint32_t M, uint32_t N, bool a_mn_major, bool b_mn_major) {
   return (1u << 4) | (2u << 7) | (2u << 10) | (uint32_t(a_mn_major) << 15) | (uint32_t(b_mn_major) << 16) |
