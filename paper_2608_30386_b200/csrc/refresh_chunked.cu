@@ -370,6 +370,15 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       {
         const int cq = lane & 7, tg = lane >> 3;
         const int c0 = warp * 32 + cq * 4, tb = tg * 8;
+        // every shared-memory read of this phase is issued before its first shared-memory write, so that
+        // the reads of later tokens do not queue behind the stores of earlier ones
+        uint2 kraw[8], qraw[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          kraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWK + (tb + j) * 256 + c0 * 2);
+          qraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + (tb + j) * 256 + c0 * 2);
+        }
+        const float4 post_prev = *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0);
         float G[8][4];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -402,7 +411,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           for (int j = 0; j < 8; ++j) G[j][i] += off;
         }
         if (tg == 0) {
-          const float4 pp = *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0);
+          const float4 pp = post_prev;
           *reinterpret_cast<float4 *>(fac_s + c0) = make_float4(ex2f((pp.x + Gm[0]) * LOG2E), ex2f((pp.y + Gm[1]) * LOG2E),
                                                                 ex2f((pp.z + Gm[2]) * LOG2E), ex2f((pp.w + Gm[3]) * LOG2E));
         } else if (tg == 1) {
@@ -412,8 +421,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int t = tb + j;
-          const uint2 kw = *reinterpret_cast<const uint2 *>(smem + OFF_RAWK + t * 256 + c0 * 2);
-          const uint2 qw = *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + t * 256 + c0 * 2);
+          const uint2 kw = kraw[j], qw = qraw[j];
           const float kf[4] = {bf16lo(kw.x), bf16hi(kw.x), bf16lo(kw.y), bf16hi(kw.y)};
           const float qf[4] = {bf16lo(qw.x), bf16hi(qw.x), bf16lo(qw.y), bf16hi(qw.y)};
           uint32_t kt[4], qt[4], kh[4];
