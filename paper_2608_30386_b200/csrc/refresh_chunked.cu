@@ -238,12 +238,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       __syncwarp();
       if (lane == 0) {
         tc_fence_after_sync();
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb)
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + kb * (64 * 128) + j * 32),
-                   desc_kmajor(sbase + OFF_KH + kb * (32 * 128) + j * 32), ID_N32, (kb | j) != 0);
+#pragma unroll 1
+        for (int kk = 0; kk < 16; ++kk)  // K = 128 in slices of 8: block kk / 4, 32 bytes per slice inside a block
+          mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
+                 desc_kmajor(sbase + OFF_KH + (kk >> 2) * (32 * 128) + (kk & 3) * 32), ID_N32, kk != 0);
         mma_commit(&misc->bar_ap);
       }
       // MMA2: S'^T [Kt;Qt]^T, the fp32 state read as a tf32 operand
@@ -251,12 +249,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       __syncwarp();
       if (lane == 0) {
         tc_fence_after_sync();
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb)
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            mma_ts(tm + COL_RO, tm + COL_S + kb * 32 + j * 8, desc_kmajor(sbase + OFF_KQ + kb * (64 * 128) + j * 32),
-                   ID_N64, (kb | j) != 0);
+#pragma unroll 1
+        for (int kk = 0; kk < 16; ++kk)
+          mma_ts(tm + COL_RO, tm + COL_S + kk * 8, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
+                 ID_N64, kk != 0);
         mma_commit(&misc->bar_ro);
       }
       // MMA3: U^T = RHS^T T^T; RHS^T is a tf32 pair (high part over R^T, low part in the A|P columns)
@@ -264,12 +260,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       __syncwarp();
       if (lane == 0) {
         tc_fence_after_sync();
-#pragma unroll
-        for (int part = 0; part < 2; ++part)
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            mma_ts(tm + COL_U, tm + (part == 0 ? COL_RO : COL_AP) + j * 8, desc_kmajor(sbase + OFF_TM + j * 32), ID_N32,
-                   (part | j) != 0);
+#pragma unroll 1
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ts(tm + COL_U, tm + (kk < 4 ? COL_RO : COL_AP) + (kk & 3) * 8, desc_kmajor(sbase + OFF_TM + (kk & 3) * 32),
+                 ID_N32, kk != 0);
         mma_commit(&misc->bar_u);
       }
       // MMA4: O^T += U^T P^T (high part of U);  MMA5: S'^T += U^T Kh (U as a pair: high in place, low over RHS^T)
@@ -278,17 +272,15 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       if (lane == 0) {
         tc_fence_after_sync();
         if (go) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            mma_ts(tm + COL_RO + 32, tm + COL_U + j * 8, desc_kmajor(sbase + OFF_PM + j * 32), ID_N32, true);
+#pragma unroll 1
+          for (int kk = 0; kk < 4; ++kk)
+            mma_ts(tm + COL_RO + 32, tm + COL_U + kk * 8, desc_kmajor(sbase + OFF_PM + kk * 32), ID_N32, true);
         }
         mma_commit(&misc->bar_o);
-#pragma unroll
-        for (int part = 0; part < 2; ++part)
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            mma_ts(tm + COL_S, tm + (part == 0 ? COL_U : COL_RO) + j * 8, desc_kmajor(sbase + OFF_KHT + j * 32), ID_N128,
-                   true);
+#pragma unroll 1
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ts(tm + COL_S, tm + (kk < 4 ? COL_U : COL_RO) + (kk & 3) * 8, desc_kmajor(sbase + OFF_KHT + (kk & 3) * 32),
+                 ID_N128, true);
         mma_commit(&misc->bar_s);
       }
       __syncwarp();
@@ -350,6 +342,22 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     }
     post_s[tid] = 0.f;  // nothing owed before the first chunk
     post_s[D + tid] = 0.f;
+    // the start state goes into TMEM as it is; the first chunk's state pass scales it like any other
+    if (n_chunks > 0) {
+#pragma unroll 1
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t s[32];
+        if (a.mode == DASC_REFRESH_CONTINUE) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) s[j] = __float_as_uint(st[(c0 + j) * D + tid]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) s[j] = 0u;
+        }
+        tmem_st32(tlane + COL_S + c0, s);
+      }
+      tmem_st_wait();
+    }
 
     for (int ch = 0; ch < n_chunks; ++ch) {
       const uint32_t par = ch & 1;
@@ -458,36 +466,22 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 
       // ---- (3) state pass: thread = value column v; scale the state to this chunk's midpoint ----
       {
-        uint32_t s[2][32];
-        auto fetch = [&](int c0, uint32_t(&dst)[32]) {
-          if (ch == 0) {
-            if (a.mode == DASC_REFRESH_CONTINUE) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) dst[j] = __float_as_uint(st[(c0 + j) * D + tid]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) dst[j] = 0u;
-            }
-          } else {
-            tmem_ld32(tlane + COL_S + c0, dst);
-          }
-        };
-        fetch(0, s[0]);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int c0 = i * 32;
-          if (ch != 0) tmem_ld_wait();
-          if (i < 3) fetch(c0 + 32, s[(i + 1) & 1]);
-          uint32_t(&cur)[32] = s[i & 1];
+        // kept as a real loop (and every other per-chunk phase as compact as possible): the chunk loop is
+        // executed once per 32 tokens by every warp, so its code size decides the instruction-fetch cost
+#pragma unroll 1
+        for (int c0 = 0; c0 < D; c0 += 32) {
+          uint32_t s[32];
+          tmem_ld32(tlane + COL_S + c0, s);
+          tmem_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             const float4 f = *reinterpret_cast<const float4 *>(fac_s + c0 + j);
-            cur[j + 0] = __float_as_uint(__uint_as_float(cur[j + 0]) * f.x);
-            cur[j + 1] = __float_as_uint(__uint_as_float(cur[j + 1]) * f.y);
-            cur[j + 2] = __float_as_uint(__uint_as_float(cur[j + 2]) * f.z);
-            cur[j + 3] = __float_as_uint(__uint_as_float(cur[j + 3]) * f.w);
+            s[j + 0] = __float_as_uint(__uint_as_float(s[j + 0]) * f.x);
+            s[j + 1] = __float_as_uint(__uint_as_float(s[j + 1]) * f.y);
+            s[j + 2] = __float_as_uint(__uint_as_float(s[j + 2]) * f.z);
+            s[j + 3] = __float_as_uint(__uint_as_float(s[j + 3]) * f.w);
           }
-          tmem_st32(tlane + COL_S + c0, cur);
+          tmem_st32(tlane + COL_S + c0, s);
         }
         tmem_st_wait();
       }
