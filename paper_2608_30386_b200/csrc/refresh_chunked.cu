@@ -378,80 +378,87 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       {
         const int cq = lane & 7, tg = lane >> 3;
         const int c0 = warp * 32 + cq * 4, tb = tg * 8;
-        // every shared-memory read of this phase is issued before its first shared-memory write, so that
-        // the reads of later tokens do not queue behind the stores of earlier ones
-        uint2 kraw[8], qraw[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          kraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWK + (tb + j) * 256 + c0 * 2);
-          qraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + (tb + j) * 256 + c0 * 2);
-        }
-        const float4 post_prev = *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0);
-        float G[8][4];
+        // pass 1: this lane's total log-decay over its 8 tokens, then the prefix over the four token groups
+        // of the warp (lanes 8 apart) and the two reference points
+        float run[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           if constexpr (KDA) {
-            const float4 gv4 = *reinterpret_cast<const float4 *>(smem + OFF_G + (tb + j) * 512 + c0 * 4);
-            G[j][0] = gv4.x; G[j][1] = gv4.y; G[j][2] = gv4.z; G[j][3] = gv4.w;
+            const float4 g4 = *reinterpret_cast<const float4 *>(smem + OFF_G + (tb + j) * 512 + c0 * 4);
+            run[0] += g4.x; run[1] += g4.y; run[2] += g4.z; run[3] += g4.w;
           } else {
             const float gs = gsc_s[par * C + tb + j];
-            G[j][0] = gs; G[j][1] = gs; G[j][2] = gs; G[j][3] = gs;
+            run[0] += gs; run[1] += gs; run[2] += gs; run[3] += gs;
           }
         }
-#pragma unroll
-        for (int j = 1; j < 8; ++j)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) G[j][i] += G[j - 1][i];
-        // prefix over the four token groups of the warp (lanes 8 apart), then the two reference points
-        float Gm[4], Gc[4];
+        const float4 post_prev = *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0);
+        float GmL[4], Gc[4], Gm[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          float incl = G[7][i];
+          float incl = run[i];
           const float own = incl;
           float x = __shfl_up_sync(0xffffffffu, incl, 8);
           if (tg >= 1) incl += x;
           x = __shfl_up_sync(0xffffffffu, incl, 16);
           if (tg >= 2) incl += x;
-          const float off = incl - own;
-          Gm[i] = __shfl_sync(0xffffffffu, incl, cq + 8);   // through token 15: the chunk midpoint
-          Gc[i] = __shfl_sync(0xffffffffu, incl, cq + 24);  // through token 31
-#pragma unroll
-          for (int j = 0; j < 8; ++j) G[j][i] += off;
+          run[i] = incl - own;                                  // log-decay accumulated before this lane's first token
+          Gm[i] = __shfl_sync(0xffffffffu, incl, cq + 8);        // through token 15: the chunk midpoint
+          Gc[i] = __shfl_sync(0xffffffffu, incl, cq + 24);       // through token 31
+          GmL[i] = Gm[i] * LOG2E;
         }
         if (tg == 0) {
-          const float4 pp = post_prev;
-          *reinterpret_cast<float4 *>(fac_s + c0) = make_float4(ex2f((pp.x + Gm[0]) * LOG2E), ex2f((pp.y + Gm[1]) * LOG2E),
-                                                                ex2f((pp.z + Gm[2]) * LOG2E), ex2f((pp.w + Gm[3]) * LOG2E));
+          *reinterpret_cast<float4 *>(fac_s + c0) =
+              make_float4(ex2f((post_prev.x + Gm[0]) * LOG2E), ex2f((post_prev.y + Gm[1]) * LOG2E),
+                          ex2f((post_prev.z + Gm[2]) * LOG2E), ex2f((post_prev.w + Gm[3]) * LOG2E));
         } else if (tg == 1) {
           *reinterpret_cast<float4 *>(post_s + par * D + c0) = make_float4(Gc[0] - Gm[0], Gc[1] - Gm[1], Gc[2] - Gm[2], Gc[3] - Gm[3]);
         }
-        uint32_t kht[4][8];
+        // pass 2: four tokens at a time (a 4 x 4 tile per lane, so that Kh can also be stored transposed).
+        // A real loop: the chunk loop runs once per 32 tokens, so code size and live registers matter.
+#pragma unroll 1
+        for (int hh = 0; hh < 2; ++hh) {
+          const int t4 = tb + hh * 4;
+          // all shared-memory reads of the tile before its first write
+          uint2 kraw[4], qraw[4];
+          float gl[4][4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int t = tb + j;
-          const uint2 kw = kraw[j], qw = qraw[j];
-          const float kf[4] = {bf16lo(kw.x), bf16hi(kw.x), bf16lo(kw.y), bf16hi(kw.y)};
-          const float qf[4] = {bf16lo(qw.x), bf16hi(qw.x), bf16lo(qw.y), bf16hi(qw.y)};
-          uint32_t kt[4], qt[4], kh[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float d = (G[j][i] - Gm[i]) * LOG2E;
-            const float e1 = ex2f(d + kLog2TruncComp), e2 = ex2f(-d);
-            kt[i] = tf32_pre(kf[i] * e1);
-            qt[i] = tf32_pre(qf[i] * a.q_scale * e1);
-            kh[i] = tf32_pre(kf[i] * e2);
-            kht[i][j] = kh[i];
+          for (int j = 0; j < 4; ++j) {
+            kraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWK + (t4 + j) * 256 + c0 * 2);
+            qraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + (t4 + j) * 256 + c0 * 2);
+            if constexpr (KDA) {
+              const float4 g4 = *reinterpret_cast<const float4 *>(smem + OFF_G + (t4 + j) * 512 + c0 * 4);
+              gl[j][0] = g4.x; gl[j][1] = g4.y; gl[j][2] = g4.z; gl[j][3] = g4.w;
+            } else {
+              const float gs = gsc_s[par * C + t4 + j];
+              gl[j][0] = gs; gl[j][1] = gs; gl[j][2] = gs; gl[j][3] = gs;
+            }
           }
-          *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, t, c0)) = make_uint4(kt[0], kt[1], kt[2], kt[3]);
-          *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, 32 + t, c0)) = make_uint4(qt[0], qt[1], qt[2], qt[3]);
-          *reinterpret_cast<uint4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_uint4(kh[0], kh[1], kh[2], kh[3]);
-        }
+          uint32_t kht[4][4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c0 + i, tb)) =
-              make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
-          *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c0 + i, tb + 4)) =
-              make_uint4(kht[i][4], kht[i][5], kht[i][6], kht[i][7]);
+          for (int j = 0; j < 4; ++j) {
+            const int t = t4 + j;
+            const uint2 kw = kraw[j], qw = qraw[j];
+            const float kf[4] = {bf16lo(kw.x), bf16hi(kw.x), bf16lo(kw.y), bf16hi(kw.y)};
+            const float qf[4] = {bf16lo(qw.x), bf16hi(qw.x), bf16lo(qw.y), bf16hi(qw.y)};
+            uint32_t kt[4], qt[4], kh[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              run[i] += gl[j][i];
+              const float d = fmaf(run[i], LOG2E, -GmL[i]);      // (G_t - G_m) log2(e)
+              const float e1 = ex2f(d + kLog2TruncComp), e2 = ex2f(-d);
+              kt[i] = tf32_pre(kf[i] * e1);
+              qt[i] = tf32_pre(qf[i] * a.q_scale * e1);
+              kh[i] = tf32_pre(kf[i] * e2);
+              kht[i][j] = kh[i];
+            }
+            *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, t, c0)) = make_uint4(kt[0], kt[1], kt[2], kt[3]);
+            *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, 32 + t, c0)) = make_uint4(qt[0], qt[1], qt[2], qt[3]);
+            *reinterpret_cast<uint4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_uint4(kh[0], kh[1], kh[2], kh[3]);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c0 + i, t4)) =
+                make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
         }
       }
       fence_smem_to_async();
