@@ -11,8 +11,8 @@
 //   S_C  = Diag(exp(G_C - G_m)) (S' + Kh^T U)
 // Referencing the decay to the midpoint keeps every exponent within half a chunk's decay.
 //
-// Mapping.  One CTA per (request, layer, value head): four compute warps and one warp that only
-// issues tensor-core work; 256 TMEM columns and about 108 KB of shared memory per CTA, so two
+// Mapping.  One CTA per (request, layer, value head): eight compute warps (two per TMEM lane quadrant,
+// each taking half of the columns) and one warp that only issues tensor-core work; 256 TMEM columns and about 108 KB of shared memory per CTA, so two
 // CTAs share an SM and one fills the other's latency gaps (every phase of a chunk depends on the
 // one before it).  The state lives in TMEM transposed, S'^T: lane = value column v, column = key
 // channel c, fp32, for the whole suffix; the tensor core reads it as a tf32 operand directly.
@@ -40,7 +40,7 @@ using namespace tc5;
 
 constexpr int C = 32;        // chunk length
 constexpr int D = 128;       // d_k = d_v
-constexpr int NC = 128;      // compute threads
+constexpr int NC = 256;      // compute threads
 constexpr int NT = NC + 32;  // + the MMA-issuing warp
 constexpr int LDX = 36;      // row pitch (floats) of the fp32 triangular work matrices
 constexpr uint32_t TMEM_COLS = 256;
@@ -93,7 +93,7 @@ constexpr float kLog2TruncComp = 5.0774e-4f;  // log2(kTruncComp)
 struct Misc {
   // tensor core -> compute warps (one tcgen05.commit each per chunk)
   uint64_t bar_ap, bar_ro, bar_u, bar_o, bar_s;
-  // compute warps -> issuing warp (128 arrivals each per chunk)
+  // compute warps -> issuing warp (256 arrivals each per chunk)
   uint64_t rdy_prep, rdy_state, rdy_rhs, rdy_u;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
@@ -114,8 +114,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// barrier among the 128 compute threads only
-__device__ __forceinline__ void sync_compute() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// barrier among the 256 compute threads only
+__device__ __forceinline__ void sync_compute() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // Bounded wait; after one time-out every later wait of this CTA returns at once.
 __device__ __forceinline__ void wait_bar(uint64_t *bar, uint32_t parity, Misc *misc, uint32_t *err) {
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     misc->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 4) {
+  if (warp == 8) {
     tmem_alloc(&misc->tmem_base, TMEM_COLS);
     tmem_relinquish();
   }
@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   constexpr uint32_t ID_N64 = idesc_tf32(128, 64, false, false);
   constexpr uint32_t ID_N128 = idesc_tf32(128, 128, false, false);
 
-  if (warp == 4) {
+  if (warp == 8) {
     // =========================== tensor-core issue warp ===========================
     for (int ch = 0; ch < n_chunks; ++ch) {
       const uint32_t par = ch & 1;
@@ -287,7 +287,9 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     }
   } else {
     // =============================== compute warps ===============================
-    const uint32_t tlane = tm + (static_cast<uint32_t>(warp * 32) << 16);  // this warp's TMEM lanes; lane index = tid
+    const int quad = warp & 3, colh = warp >> 2;                           // TMEM lane quadrant, column half
+    const uint32_t tlane = tm + (static_cast<uint32_t>(quad * 32) << 16);  // this warp's TMEM lanes
+    const int vrow = quad * 32 + lane;                                     // the TMEM lane this thread owns
     constexpr float LOG2E = 1.4426950408889634f;
     PT_DECL
 
@@ -340,16 +342,15 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       asm volatile("cp.async.commit_group;" ::: "memory");
       store_scalar(0, load_scalar(0));
     }
-    post_s[tid] = 0.f;  // nothing owed before the first chunk
-    post_s[D + tid] = 0.f;
+    post_s[tid] = 0.f;  // [2][128]: nothing owed before the first chunk
     // the start state goes into TMEM as it is; the first chunk's state pass scales it like any other
     if (n_chunks > 0) {
 #pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
+      for (int c0 = colh * 64; c0 < colh * 64 + 64; c0 += 32) {
         uint32_t s[32];
         if (a.mode == DASC_REFRESH_CONTINUE) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) s[j] = __float_as_uint(st[(c0 + j) * D + tid]);
+          for (int j = 0; j < 32; ++j) s[j] = __float_as_uint(st[(c0 + j) * D + vrow]);
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j) s[j] = 0u;
@@ -374,92 +375,77 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       const float scalar_next = more ? load_scalar(ch + 1) : 0.f;  // in flight during the chunk
       PT(0);
 
-      // ---- (2) prep: warp = block of 32 channels; lane = (4 adjacent channels, 8 consecutive tokens) ----
+      // ---- (2) prep: warp = (block of 32 channels, half of the tokens); lane = (4 adjacent channels, 4 consecutive
+      //          tokens), a 4 x 4 tile, so that Kh can also be stored transposed.  The midpoint is the end of the
+      //          first half: first-half exponents are (local sum - the half's total), second-half exponents the
+      //          local sums themselves. ----
       {
-        const int cq = lane & 7, tg = lane >> 3;
-        const int c0 = warp * 32 + cq * 4, tb = tg * 8;
-        // pass 1: this lane's total log-decay over its 8 tokens, then the prefix over the four token groups
-        // of the warp (lanes 8 apart) and the two reference points
-        float run[4] = {0.f, 0.f, 0.f, 0.f};
+        const int cq = lane & 7, tg = lane >> 3, half = warp >> 2;
+        const int c0 = (warp & 3) * 32 + cq * 4, t4 = half * 16 + tg * 4;
+        // all shared-memory reads of the tile before its first write
+        uint2 kraw[4], qraw[4];
+        float gl[4][4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < 4; ++j) {
+          kraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWK + (t4 + j) * 256 + c0 * 2);
+          qraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + (t4 + j) * 256 + c0 * 2);
           if constexpr (KDA) {
-            const float4 g4 = *reinterpret_cast<const float4 *>(smem + OFF_G + (tb + j) * 512 + c0 * 4);
-            run[0] += g4.x; run[1] += g4.y; run[2] += g4.z; run[3] += g4.w;
+            const float4 g4 = *reinterpret_cast<const float4 *>(smem + OFF_G + (t4 + j) * 512 + c0 * 4);
+            gl[j][0] = g4.x; gl[j][1] = g4.y; gl[j][2] = g4.z; gl[j][3] = g4.w;
           } else {
-            const float gs = gsc_s[par * C + tb + j];
-            run[0] += gs; run[1] += gs; run[2] += gs; run[3] += gs;
+            const float gs = gsc_s[par * C + t4 + j];
+            gl[j][0] = gs; gl[j][1] = gs; gl[j][2] = gs; gl[j][3] = gs;
           }
         }
         const float4 post_prev = *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0);
-        float GmL[4], Gc[4], Gm[4];
+        // this lane's total, the prefix over the four token groups of the warp (lanes 8 apart), the half's total
+        float run[4], refL[4], tot[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          float incl = run[i];
+          float incl = gl[0][i] + gl[1][i] + gl[2][i] + gl[3][i];
           const float own = incl;
           float x = __shfl_up_sync(0xffffffffu, incl, 8);
           if (tg >= 1) incl += x;
           x = __shfl_up_sync(0xffffffffu, incl, 16);
           if (tg >= 2) incl += x;
-          run[i] = incl - own;                                  // log-decay accumulated before this lane's first token
-          Gm[i] = __shfl_sync(0xffffffffu, incl, cq + 8);        // through token 15: the chunk midpoint
-          Gc[i] = __shfl_sync(0xffffffffu, incl, cq + 24);       // through token 31
-          GmL[i] = Gm[i] * LOG2E;
+          run[i] = incl - own;                               // accumulated before this lane's first token
+          tot[i] = __shfl_sync(0xffffffffu, incl, cq + 24);   // the half's total
+          refL[i] = half == 0 ? tot[i] * LOG2E : 0.f;
         }
         if (tg == 0) {
-          *reinterpret_cast<float4 *>(fac_s + c0) =
-              make_float4(ex2f((post_prev.x + Gm[0]) * LOG2E), ex2f((post_prev.y + Gm[1]) * LOG2E),
-                          ex2f((post_prev.z + Gm[2]) * LOG2E), ex2f((post_prev.w + Gm[3]) * LOG2E));
-        } else if (tg == 1) {
-          *reinterpret_cast<float4 *>(post_s + par * D + c0) = make_float4(Gc[0] - Gm[0], Gc[1] - Gm[1], Gc[2] - Gm[2], Gc[3] - Gm[3]);
+          if (half == 0)
+            *reinterpret_cast<float4 *>(fac_s + c0) =
+                make_float4(ex2f((post_prev.x + tot[0]) * LOG2E), ex2f((post_prev.y + tot[1]) * LOG2E),
+                            ex2f((post_prev.z + tot[2]) * LOG2E), ex2f((post_prev.w + tot[3]) * LOG2E));
+          else
+            *reinterpret_cast<float4 *>(post_s + par * D + c0) = make_float4(tot[0], tot[1], tot[2], tot[3]);  // G_C - G_m
         }
-        // pass 2: four tokens at a time (a 4 x 4 tile per lane, so that Kh can also be stored transposed).
-        // A real loop: the chunk loop runs once per 32 tokens, so code size and live registers matter.
-#pragma unroll 1
-        for (int hh = 0; hh < 2; ++hh) {
-          const int t4 = tb + hh * 4;
-          // all shared-memory reads of the tile before its first write
-          uint2 kraw[4], qraw[4];
-          float gl[4][4];
+        uint32_t kht[4][4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            kraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWK + (t4 + j) * 256 + c0 * 2);
-            qraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + (t4 + j) * 256 + c0 * 2);
-            if constexpr (KDA) {
-              const float4 g4 = *reinterpret_cast<const float4 *>(smem + OFF_G + (t4 + j) * 512 + c0 * 4);
-              gl[j][0] = g4.x; gl[j][1] = g4.y; gl[j][2] = g4.z; gl[j][3] = g4.w;
-            } else {
-              const float gs = gsc_s[par * C + t4 + j];
-              gl[j][0] = gs; gl[j][1] = gs; gl[j][2] = gs; gl[j][3] = gs;
-            }
+        for (int j = 0; j < 4; ++j) {
+          const int t = t4 + j;
+          const uint2 kw = kraw[j], qw = qraw[j];
+          const float kf[4] = {bf16lo(kw.x), bf16hi(kw.x), bf16lo(kw.y), bf16hi(kw.y)};
+          const float qf[4] = {bf16lo(qw.x), bf16hi(qw.x), bf16lo(qw.y), bf16hi(qw.y)};
+          uint32_t kt[4], qt[4], kh[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            run[i] += gl[j][i];
+            const float d = fmaf(run[i], LOG2E, -refL[i]);      // (G_t - G_m) log2(e)
+            const float e1 = ex2f(d + kLog2TruncComp), e2 = ex2f(-d);
+            kt[i] = tf32_pre(kf[i] * e1);
+            qt[i] = tf32_pre(qf[i] * a.q_scale * e1);
+            kh[i] = tf32_pre(kf[i] * e2);
+            kht[i][j] = kh[i];
           }
-          uint32_t kht[4][4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int t = t4 + j;
-            const uint2 kw = kraw[j], qw = qraw[j];
-            const float kf[4] = {bf16lo(kw.x), bf16hi(kw.x), bf16lo(kw.y), bf16hi(kw.y)};
-            const float qf[4] = {bf16lo(qw.x), bf16hi(qw.x), bf16lo(qw.y), bf16hi(qw.y)};
-            uint32_t kt[4], qt[4], kh[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              run[i] += gl[j][i];
-              const float d = fmaf(run[i], LOG2E, -GmL[i]);      // (G_t - G_m) log2(e)
-              const float e1 = ex2f(d + kLog2TruncComp), e2 = ex2f(-d);
-              kt[i] = tf32_pre(kf[i] * e1);
-              qt[i] = tf32_pre(qf[i] * a.q_scale * e1);
-              kh[i] = tf32_pre(kf[i] * e2);
-              kht[i][j] = kh[i];
-            }
-            *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, t, c0)) = make_uint4(kt[0], kt[1], kt[2], kt[3]);
-            *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, 32 + t, c0)) = make_uint4(qt[0], qt[1], qt[2], qt[3]);
-            *reinterpret_cast<uint4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_uint4(kh[0], kh[1], kh[2], kh[3]);
-          }
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c0 + i, t4)) =
-                make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
+          *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, t, c0)) = make_uint4(kt[0], kt[1], kt[2], kt[3]);
+          *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, 32 + t, c0)) = make_uint4(qt[0], qt[1], qt[2], qt[3]);
+          *reinterpret_cast<uint4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_uint4(kh[0], kh[1], kh[2], kh[3]);
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c0 + i, t4)) =
+              make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
       }
       fence_smem_to_async();
       tc_fence_before_sync();
@@ -471,12 +457,12 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       asm volatile("cp.async.commit_group;" ::: "memory");
       PT(1);
 
-      // ---- (3) state pass: thread = value column v; scale the state to this chunk's midpoint ----
+      // ---- (3) state pass: thread = (value column v, half of the channels); scale the state to this chunk's midpoint ----
       {
         // kept as a real loop (and every other per-chunk phase as compact as possible): the chunk loop is
         // executed once per 32 tokens by every warp, so its code size decides the instruction-fetch cost
 #pragma unroll 1
-        for (int c0 = 0; c0 < D; c0 += 32) {
+        for (int c0 = colh * 64; c0 < colh * 64 + 64; c0 += 32) {
           uint32_t s[32];
           tmem_ld32(tlane + COL_S + c0, s);
           tmem_ld_wait();
@@ -564,10 +550,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       sync_compute();
       PT(4);
       {
-        // T (lower triangle of X, unit diagonal) -> tf32 operand tile; 8 elements per thread
-        const int t = tid >> 2, i0 = (tid & 3) * 8;
+        // T (lower triangle of X, unit diagonal) -> tf32 operand tile; 4 elements per thread
+        const int t = tid >> 3, i0 = (tid & 7) * 4;
 #pragma unroll
-        for (int j = 0; j < 8; j += 4) {
+        for (int j = 0; j < 4; j += 4) {
           const float4 xv = *reinterpret_cast<const float4 *>(Xm + t * LDX + i0 + j);
           uint4 o;
           o.x = (i0 + j + 0 <= t) ? tf32_pre(xv.x) : 0u;
@@ -587,18 +573,19 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       sync_compute();
       PT(6);
       {
-        uint32_t x[32], lo[32];
-        tmem_ld32(tlane + COL_RO, x);
+        const int tb = colh * 16;
+        uint32_t x[16], lo[16];
+        tmem_ld16(tlane + COL_RO + tb, x);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float vv = __bfloat162float(Vs[j * D + tid]);
-          const float rhs = beta_c[j] * (vv - __uint_as_float(x[j]));
+        for (int j = 0; j < 16; ++j) {
+          const float vv = __bfloat162float(Vs[(tb + j) * D + vrow]);
+          const float rhs = beta_c[tb + j] * (vv - __uint_as_float(x[j]));
           x[j] = to_tf32(rhs);
           lo[j] = tf32_pre(rhs - __uint_as_float(x[j]));
         }
-        tmem_st32(tlane + COL_RO, x);
-        tmem_st32(tlane + COL_AP, lo);
+        tmem_st16(tlane + COL_RO + tb, x);
+        tmem_st16(tlane + COL_AP + tb, lo);
         tmem_st_wait();
       }
       tc_fence_before_sync();
@@ -613,17 +600,18 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       tc_fence_after_sync();
       PT(8);
       {
-        uint32_t x[32], lo[32];
-        tmem_ld32(tlane + COL_U, x);
+        const int tb = colh * 16;
+        uint32_t x[16], lo[16];
+        tmem_ld16(tlane + COL_U + tb, x);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
+        for (int j = 0; j < 16; ++j) {
           const float u = __uint_as_float(x[j]);
           x[j] = to_tf32(u);
           lo[j] = tf32_pre(u - __uint_as_float(x[j]));
         }
-        tmem_st32(tlane + COL_U, x);
-        tmem_st32(tlane + COL_RO, lo);
+        tmem_st16(tlane + COL_U + tb, x);
+        tmem_st16(tlane + COL_RO + tb, lo);
         tmem_st_wait();
       }
       tc_fence_before_sync();
@@ -635,14 +623,15 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       tc_fence_after_sync();
       PT(10);
       if (go) {
-        uint32_t x[32];
-        tmem_ld32(tlane + COL_RO + 32, x);
+        const int tb = colh * 16;
+        uint32_t x[16];
+        tmem_ld16(tlane + COL_RO + 32 + tb, x);
         tmem_ld_wait();
         if constexpr (sizeof(OT) == 2) {
           // through shared memory (the Kt/Qt tile is free now) so that global stores are 16 bytes wide
           __nv_bfloat16 *Os = reinterpret_cast<__nv_bfloat16 *>(smem + OFF_KQ);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) Os[j * D + tid] = __float2bfloat16_rn(__uint_as_float(x[j]));
+          for (int j = 0; j < 16; ++j) Os[(tb + j) * D + vrow] = __float2bfloat16_rn(__uint_as_float(x[j]));
           sync_compute();
           for (int i = tid; i < ntok * 16; i += NC) {
             const int t = i >> 4, j = i & 15;
@@ -651,8 +640,8 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           }
         } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (j < ntok) go[(t0 + j) * v_stride + tid] = __uint_as_float(x[j]);
+          for (int j = 0; j < 16; ++j)
+            if (tb + j < ntok) go[(t0 + tb + j) * v_stride + vrow] = __uint_as_float(x[j]);
         }
       }
       store_scalar(ch + 1, scalar_next);
@@ -663,14 +652,14 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 
     // ---- final state: the factor still owed, then write back ----
     if (n_chunks > 0) wait_bar(&misc->bar_s, (n_chunks - 1) & 1, misc, err);
-    fac_s[tid] = ex2f(post_s[((n_chunks + 1) & 1) * D + tid] * LOG2E);
+    if (tid < D) fac_s[tid] = ex2f(post_s[((n_chunks + 1) & 1) * D + tid] * LOG2E);
     sync_compute();
     tc_fence_after_sync();
     {
       const uint8_t *keep = a.row_keep + static_cast<int64_t>(layer) * a.rows_per_layer + static_cast<int64_t>(h) * D;
       const bool merge = a.mode != DASC_REFRESH_CONTINUE;
 #pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
+      for (int c0 = colh * 64; c0 < colh * 64 + 64; c0 += 32) {
         uint32_t s[32];
         if (n_chunks > 0) {
           tmem_ld32(tlane + COL_S + c0, s);
@@ -682,7 +671,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const int c = c0 + j;
-          if (!merge || !keep[c]) st[c * D + tid] = __uint_as_float(s[j]) * fac_s[c];
+          if (!merge || !keep[c]) st[c * D + vrow] = __uint_as_float(s[j]) * fac_s[c];
         }
       }
     }
@@ -691,7 +680,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 4) tmem_dealloc(tm, TMEM_COLS);
+  if (warp == 8) tmem_dealloc(tm, TMEM_COLS);
 }
 
 template <bool KDA, typename OT>
