@@ -40,7 +40,8 @@ import torch  # noqa: E402
 D = 128
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 TF32_OVER_BF16 = 0.489        # nominal dense 1.1 : 2.25
-CHUNKED_FLOPS_PER_TOKEN_HEAD = 163840   # tf32 flops the chunked kernel issues per (token, head)
+CHUNKED_FLOPS_PER_TOKEN_HEAD = 188416   # tf32 flops the chunked kernel issues per (token, head): 32-token chunks,
+                                        # MMA1 padded to M = 128, hi/lo pairs in MMA3 and MMA5
 
 CONFIGS = {
     1: dict(name="kda_serving", kind="KDA", L=24, H_v=32, H_k=32, n_req=64, keep=0.38, rate_lo=1e-3, suffix=256, seed=1),

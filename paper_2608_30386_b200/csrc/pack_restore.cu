@@ -8,7 +8,16 @@
 
 namespace {
 
-constexpr int kThreads = 256;
+#ifndef DASC_COPY_THREADS
+#define DASC_COPY_THREADS 256
+#endif
+#ifndef DASC_PACK_UNROLL
+#define DASC_PACK_UNROLL 4
+#endif
+#ifndef DASC_RESTORE_UNROLL
+#define DASC_RESTORE_UNROLL 4
+#endif
+constexpr int kThreads = DASC_COPY_THREADS;  // tuning knobs; defaults = best of a sweep over {128..1024} x {2..16}
 
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
   uint4 v;
@@ -90,8 +99,8 @@ __global__ void __launch_bounds__(kThreads) restore_kernel(const uint4 *__restri
   }
 }
 
-constexpr int kPackUnroll = 8;
-constexpr int kRestoreUnroll = 8;
+constexpr int kPackUnroll = DASC_PACK_UNROLL;
+constexpr int kRestoreUnroll = DASC_RESTORE_UNROLL;
 
 }  // namespace
 
