@@ -211,10 +211,13 @@ dasc_status_t dasc_restore(const dasc_plan_t *plan, const float *pool_base, int6
  *   copied into the stored state, retained units keep their stored values.
  *
  * algo SEQUENTIAL is exact fp32 arithmetic token by token and accepts any g <= 0.
- * algo CHUNKED processes 64-token chunks on the tensor cores; it needs
- *   d_k = d_v = 128 and, for every 32 consecutive tokens and every channel,
- *   sum |g| <= 80 (decay factors are formed relative to the chunk midpoint in
- *   fp32).  AUTO picks CHUNKED when the shape allows it.
+ * algo CHUNKED processes 32-token chunks on the tensor cores (tf32 operands,
+ *   fp32 accumulation and fp32 state); it needs d_k = d_v = 128, bf16 q/k/v
+ *   and, for every 16 consecutive tokens and every channel, sum |g| <= 80
+ *   (decay factors are formed relative to the chunk midpoint in fp32); it
+ *   returns DASC_ERR_SHAPE otherwise.  AUTO picks CHUNKED when shape
+ *   and dtype allow it and SEQUENTIAL when they do not; the bound on g is
+ *   the caller's to know.
  *
  * workspace: DEVICE scratch of at least dasc_refresh_workspace_bytes(), 256-byte
  *   aligned, private to this call until it completes; may be NULL when that
