@@ -43,6 +43,13 @@ TF32_OVER_BF16 = 0.489        # nominal dense 1.1 : 2.25
 CHUNKED_FLOPS_PER_TOKEN_HEAD = 188416   # tf32 flops the chunked kernel issues per (token, head): 32-token chunks,
                                         # MMA1 padded to M = 128, hi/lo pairs in MMA3 and MMA5
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes, from one ncu full-set capture of
+# the KDA serving workload at 8 requests and a 128-token suffix (a full-size launch is too large to capture); every
+# request and token moves the same bytes, so traffic grows in proportion and a full launch is scaled by its units.
+# Below 1.0 = lines still dirty in L2 when the kernel ended, not skipped work.
+NCU_TRAFFIC_OVER_ALGORITHMIC = {"pack": 254.99e6 / 306.12e6, "restore": 499.80e6 / 555.71e6,
+                                "refresh_chunked": 1.9815e9 / 2.0164e9}
+
 CONFIGS = {
     1: dict(name="kda_serving", kind="KDA", L=24, H_v=32, H_k=32, n_req=64, keep=0.38, rate_lo=1e-3, suffix=256, seed=1),
     2: dict(name="gdn_headwise", kind="GDN", L=36, H_v=32, H_k=16, n_req=128, keep=0.5, rate_lo=1e-4, suffix=256, seed=2),
@@ -432,6 +439,15 @@ def main():
                     "frac_of_fp32_alu": refresh_tflops / alu_tflops, "tflops_tf32_issued": tf32_issued,
                     "tf32_peak": TF32_OVER_BF16 * tf, "frac_of_tf32_tensor": tf32_issued / (TF32_OVER_BF16 * tf)},
     }
+    if c["name"] == "kda_serving":      # the workload the capture was made on
+        rl["pack"]["traffic"] = NCU_TRAFFIC_OVER_ALGORITHMIC["pack"] * pack_bytes
+        rl["restore"]["traffic"] = NCU_TRAFFIC_OVER_ALGORITHMIC["restore"] * restore_bytes
+        if args.algo != "sequential":       # auto picks the chunked kernel for this shape
+            rl["refresh"]["traffic"] = NCU_TRAFFIC_OVER_ALGORITHMIC["refresh_chunked"] * refresh_bytes / n_groups
+    rl["refresh"]["launches_per_step"] = n_groups
+    rl["refresh"]["algorithmic_bytes_per_launch"] = refresh_bytes / n_groups
+    rl["pack"]["algorithmic_bytes_per_launch"] = pack_bytes
+    rl["restore"]["algorithmic_bytes_per_launch"] = restore_bytes
     dominant = max((("pack", t_pack), ("restore", t_restore), ("refresh", t_refresh)), key=lambda x: x[1])[0]
     roofline = dict(rl[dominant])
     roofline["kernel"] = dominant
