@@ -59,7 +59,9 @@ CONFIGS = {
 
 
 def workload_name(c):
-    return (f"{c['name']}_{c['L']}x{c['H_v']}x{D}x{D}_fp32_{c['n_req']}req_keep{c['keep']}_suffix{c['suffix']}_bf16")
+    codec = "_int8pool" if c.get("codec") == "int8" else ""
+    return (f"{c['name']}_{c['L']}x{c['H_v']}x{D}x{D}_fp32_{c['n_req']}req_keep{c['keep']}_suffix{c['suffix']}_bf16"
+            f"{codec}")
 
 
 def peaks():
@@ -150,13 +152,19 @@ def oracle_leg(c, sample_req=4, sample_units=64):
     pool = np.zeros((sample_req, slot), np.float32)
     out = np.empty_like(state)
     ids = np.arange(sample_req, dtype=np.int32)
+    int8 = c.get("codec") == "int8"
+    slot_bytes = slot // D * (D + 4) if int8 else slot * 4
     t0 = time.perf_counter()
     oracle.pack(oplan.mask, unit_words, state, dense, L * dense, ids, pool, slot, ids)
+    if int8:
+        codes, scales = oracle.int8_quantize(pool.reshape(-1, D))
     t1 = time.perf_counter()
+    if int8:
+        pool = oracle.int8_dequantize(codes, scales).reshape(sample_req, slot)
     oracle.restore(oplan.mask, unit_words, pool, slot, ids, out, dense, L * dense, ids)
     t2 = time.perf_counter()
-    pack_bytes = 2 * sample_req * slot * 4
-    restore_bytes = sample_req * (slot + L * dense) * 4
+    pack_bytes = sample_req * (slot * 4 + slot_bytes)
+    restore_bytes = sample_req * (slot_bytes + L * dense * 4)
     # refresh sample: whole layers of one request (sample_units (request, layer, head) units), 256 tokens
     Ls = max(1, sample_units // H_v)
     n_tok = min(c["suffix"], 256)
@@ -239,6 +247,8 @@ def main():
     ap.add_argument("--suffix", type=int, default=None, help="refresh suffix length (config 3: 256, 1024, 4096)")
     ap.add_argument("--keep", type=float, default=None, help="keep ratio (0.25, 0.38, 0.5, 1.0 in the sweep)")
     ap.add_argument("--layer-group", type=int, default=None, help="layers of token streams resident at once")
+    ap.add_argument("--codec", default="fp32", choices=["fp32", "int8"],
+                    help="checkpoint pool format: fp32 bit copies, or the Appendix D INT8 codec fused into pack/restore")
     args = ap.parse_args()
     c = dict(CONFIGS[args.config])
     if args.requests is not None:
@@ -247,6 +257,7 @@ def main():
         c["suffix"] = args.suffix
     if args.keep is not None:
         c["keep"] = args.keep
+    c["codec"] = args.codec
     if args.impl == "reference":
         run_reference(args, c)
         return
@@ -281,7 +292,12 @@ def main():
     state = synth.states(dgen, (L, N_REQ, dense), dev)
     active = torch.empty_like(state)
     slot = int(plan.slot_floats)
-    pool = torch.empty((N_REQ, slot), device=dev)
+    int8 = args.codec == "int8"
+    # bytes of one checkpoint slot in the pool: fp32 rows, or int8 codes + one fp32 scale per row
+    slot_bytes = dasc.dasc_int8_slot_bytes(plan) if int8 else slot * 4
+    pool = torch.empty((N_REQ, slot_bytes), dtype=torch.uint8, device=dev) if int8 else torch.empty((N_REQ, slot), device=dev)
+    do_pack = dasc.dasc_pack_int8 if int8 else dasc.dasc_pack
+    do_restore = dasc.dasc_restore_int8 if int8 else dasc.dasc_restore
     ids = torch.arange(N_REQ, dtype=torch.int32, device=dev)
     slots = torch.randperm(N_REQ, generator=gen).to(torch.int32).to(dev)
     T = N_REQ * SUFFIX
@@ -300,8 +316,8 @@ def main():
     ws_bytes = dasc.dasc_refresh_workspace_bytes(plan, N_REQ, group, algo)
     ws = torch.zeros(max(ws_bytes, 256), dtype=torch.uint8, device=dev) if ws_bytes else None
 
-    pack_bytes = 2 * N_REQ * slot * 4
-    restore_bytes = N_REQ * (slot + L * dense) * 4
+    pack_bytes = N_REQ * (slot * 4 + slot_bytes)
+    restore_bytes = N_REQ * (slot_bytes + L * dense * 4)
     token_heads = N_REQ * L * H_v * SUFFIX
     refresh_bytes = token_heads * token_bytes_per_head(kda, H_v, H_k) + 2 * N_REQ * L * dense * 4  # + state in and out
     refresh_flops_min = token_heads * 7 * D * D              # token-by-token recurrence, incl. decay and read-out
@@ -312,10 +328,10 @@ def main():
     def step(ev=None):
         if ev:
             ev[0].record(stream)
-        dasc.dasc_pack(plan, state, layer_stride, req_stride, ids, pool, slots)
+        do_pack(plan, state, layer_stride, req_stride, ids, pool, slots)
         if ev:
             ev[1].record(stream)
-        dasc.dasc_restore(plan, pool, slots, active, layer_stride, req_stride, ids)
+        do_restore(plan, pool, slots, active, layer_stride, req_stride, ids)
         if ev:
             ev[2].record(stream)
         for gi in range(n_groups):
@@ -362,12 +378,13 @@ def main():
         h_state = torch.empty((L, n_e, dense), dtype=torch.float32).pin_memory()
         h_state.copy_(state[:, :n_e])
         host_streams = [x[:ge, :Te].contiguous().cpu().pin_memory() for x in (q, k, v, g, beta)]
-        h_pool = torch.empty((n_e, slot), dtype=torch.float32).pin_memory()
+        pool_shape, pool_dtype = ((n_e, slot_bytes), torch.uint8) if int8 else ((n_e, slot), torch.float32)
+        h_pool = torch.empty(pool_shape, dtype=pool_dtype).pin_memory()
         h_out = torch.empty((L, n_e, dense), dtype=torch.float32).pin_memory()
         h_o = torch.empty((ge, Te, H_v, D), dtype=torch.bfloat16).pin_memory()
         d_state = torch.empty((L, n_e, dense), device=dev)
         d_active = torch.empty_like(d_state)
-        d_pool = torch.empty((n_e, slot), device=dev)
+        d_pool = torch.empty(pool_shape, dtype=pool_dtype, device=dev)
         d_streams = [torch.empty(x.shape, dtype=x.dtype, device=dev) for x in host_streams]
         d_o = torch.empty((ge, Te, H_v, D), dtype=torch.bfloat16, device=dev)
         cu_e = synth.uniform_cu_seqlens(n_e, SUFFIX).to(dev)
@@ -377,8 +394,8 @@ def main():
         def e2e_step(ev):
             ev[0].record(stream)
             d_state.copy_(h_state, non_blocking=True)
-            dasc.dasc_pack(plan, d_state, ls_e, dense, ids_e, d_pool, ids_e)
-            dasc.dasc_restore(plan, d_pool, ids_e, d_active, ls_e, dense, ids_e)
+            do_pack(plan, d_state, ls_e, dense, ids_e, d_pool, ids_e)
+            do_restore(plan, d_pool, ids_e, d_active, ls_e, dense, ids_e)
             h_pool.copy_(d_pool, non_blocking=True)
             ev[1].record(stream)
             for gi in range(L // ge):                        # every layer group: its streams in, its outputs out
@@ -403,9 +420,9 @@ def main():
         if dist:
             dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         t_copy, t_ref = tt.tolist()
-        e_bytes = (2 * n_e * slot + n_e * (slot + L * dense)) * 4
+        e_bytes = n_e * (slot * 4 + slot_bytes) + n_e * (slot_bytes + L * dense * 4)
         h2d = h_state.numel() * 4 + (L // ge) * sum(x.numel() * x.element_size() for x in host_streams)
-        d2h = h_pool.numel() * 4 + h_out.numel() * 4 + (L // ge) * h_o.numel() * 2
+        d2h = h_pool.numel() * h_pool.element_size() + h_out.numel() * 4 + (L // ge) * h_o.numel() * 2
         e2e = {"value": world * e_bytes / (t_copy * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "requests_per_step": n_e,
                "refresh_tokens_per_s": world * Te / (t_ref * 1e-3), "ms_pack_restore": t_copy, "ms_refresh": t_ref,
@@ -439,7 +456,7 @@ def main():
                     "frac_of_fp32_alu": refresh_tflops / alu_tflops, "tflops_tf32_issued": tf32_issued,
                     "tf32_peak": TF32_OVER_BF16 * tf, "frac_of_tf32_tensor": tf32_issued / (TF32_OVER_BF16 * tf)},
     }
-    if c["name"] == "kda_serving":      # the workload the capture was made on
+    if c["name"] == "kda_serving" and not int8:      # the workload the capture was made on
         rl["pack"]["traffic"] = NCU_TRAFFIC_OVER_ALGORITHMIC["pack"] * pack_bytes
         rl["restore"]["traffic"] = NCU_TRAFFIC_OVER_ALGORITHMIC["restore"] * restore_bytes
         if args.algo != "sequential":       # auto picks the chunked kernel for this shape
@@ -456,7 +473,7 @@ def main():
         "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_total,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(c), "kind": c["kind"], "layers": L, "v_heads": H_v, "k_heads": H_k, "d_k": D,
-                   "d_v": D, "requests": N_REQ, "keep_ratio": c["keep"], "suffix_tokens": SUFFIX, "refresh_algo": args.algo,
+                   "d_v": D, "requests": N_REQ, "keep_ratio": c["keep"], "codec": args.codec, "suffix_tokens": SUFFIX, "refresh_algo": args.algo,
                    "stream_layers_resident": group,
                    "l2": "inputs larger than L2 (GiBs of states and token streams per step); no flush needed",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},

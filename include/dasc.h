@@ -184,6 +184,37 @@ dasc_status_t dasc_restore(const dasc_plan_t *plan, const float *pool_base, int6
                            void *cuda_stream);
 
 /*
+ * INT8 checkpoint codec fused into the Store / Load copies (Appendix D, Eq. 10).
+ * A row is the d_v values of one (layer, head, key channel) tuple; rows are the
+ * plan's retained rows in ragged order (a retained GDN head contributes its d_k
+ * rows).  Per row, in fp32 arithmetic:
+ *     a = max_v |S|,  s = max(a, 1e-8) / 127,
+ *     q = clip(round(S / s), -127, 127)     (round to nearest, ties to even)
+ * and on load  S_hat = q * s  (one fp32 multiply); omitted rows are zero-filled
+ * exactly as in dasc_restore.  Values must be finite (the formula says nothing
+ * about NaN or infinity; their codes are unspecified).
+ *
+ * Slot layout in BYTES: [packed_rows][d_v] int8 codes, then [packed_rows] fp32
+ * scales, packed_rows = sum_r for KDA and sum_r * d_k for GDN.
+ *   dasc_int8_slot_bytes  bytes of one slot, rounded up to a multiple of 16.
+ *   pool_base             DEVICE, 16-byte aligned.
+ *   slot_stride_bytes     bytes between slots, multiple of 16, >= the slot
+ *                         size; 0 = the slot size.
+ * Everything else (state pointer, strides in floats, index arrays, n_pairs,
+ * distinctness, stream, errors) as for dasc_pack / dasc_restore.
+ * d_v must be a power of two between 4 and 128 (DASC_ERR_SHAPE otherwise).
+ */
+dasc_status_t dasc_int8_slot_bytes(const dasc_plan_t *plan, size_t *out);
+dasc_status_t dasc_pack_int8(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride,
+                             int64_t req_stride, const int32_t *src_req, void *pool_base,
+                             int64_t slot_stride_bytes, const int32_t *dst_slot, int32_t n_pairs,
+                             void *cuda_stream);
+dasc_status_t dasc_restore_int8(const dasc_plan_t *plan, const void *pool_base,
+                                int64_t slot_stride_bytes, const int32_t *src_slot,
+                                float *state_base, int64_t layer_stride, int64_t req_stride,
+                                const int32_t *dst_req, int32_t n_pairs, void *cuda_stream);
+
+/*
  * Suffix refresh: replay the gated delta rule (Eq. 1, transposed orientation)
  *     S_t = (I - beta_t k_t k_t^T) Diag(alpha_t) S_{t-1} + beta_t k_t v_t^T,   alpha_t = exp(g_t)
  *     o_t = q_scale * S_t^T q_t

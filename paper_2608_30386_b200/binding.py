@@ -29,6 +29,7 @@ OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_WORKSP
 EXPORTS = (
     "dasc_plan", "dasc_plan_destroy", "dasc_plan_info", "dasc_plan_horizon", "dasc_plan_mask",
     "dasc_plan_window", "dasc_plan_layer_counts", "dasc_plan_layer_offsets", "dasc_pack", "dasc_restore",
+    "dasc_int8_slot_bytes", "dasc_pack_int8", "dasc_restore_int8",
     "dasc_refresh_workspace_bytes", "dasc_refresh", "dasc_refresh_status", "dasc_refresh_static",
     "dasc_status_string", "dasc_version",
 )
@@ -89,6 +90,9 @@ def lib() -> C.CDLL:
                                 C.c_void_p, C.c_int32, C.c_void_p]
         L.dasc_restore.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                    C.c_void_p, C.c_int32, C.c_void_p]
+        L.dasc_int8_slot_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
+        L.dasc_pack_int8.argtypes = L.dasc_pack.argtypes
+        L.dasc_restore_int8.argtypes = L.dasc_restore.argtypes
         L.dasc_refresh_workspace_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]
         L.dasc_refresh.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int64,
@@ -216,6 +220,29 @@ def dasc_restore(plan: Plan, pool: torch.Tensor, src_slot: torch.Tensor, state: 
     """Scatter pool slots ``src_slot`` into the dense states ``dst_req``; omitted units become +0.0."""
     _check(lib().dasc_restore(plan.handle, _ptr(pool), slot_stride, _ptr(src_slot), _ptr(state), layer_stride,
                               req_stride, _ptr(dst_req), int(src_slot.numel()), _stream_ptr(stream)), "dasc_restore")
+
+
+def dasc_int8_slot_bytes(plan: Plan) -> int:
+    """Bytes of one INT8 slot: codes [packed_rows][d_v] then fp32 scales [packed_rows], rounded up to 16."""
+    out = C.c_size_t()
+    _check(lib().dasc_int8_slot_bytes(plan.handle, C.byref(out)), "dasc_int8_slot_bytes")
+    return int(out.value)
+
+
+def dasc_pack_int8(plan: Plan, state: torch.Tensor, layer_stride: int, req_stride: int, src_req: torch.Tensor,
+                   pool: torch.Tensor, dst_slot: torch.Tensor, slot_stride_bytes: int = 0, stream=None):
+    """Like ``dasc_pack`` with the Appendix D quantiser fused in; ``pool`` is a byte (uint8) tensor."""
+    _check(lib().dasc_pack_int8(plan.handle, _ptr(state), layer_stride, req_stride, _ptr(src_req), _ptr(pool),
+                                slot_stride_bytes, _ptr(dst_slot), int(src_req.numel()), _stream_ptr(stream)),
+           "dasc_pack_int8")
+
+
+def dasc_restore_int8(plan: Plan, pool: torch.Tensor, src_slot: torch.Tensor, state: torch.Tensor, layer_stride: int,
+                      req_stride: int, dst_req: torch.Tensor, slot_stride_bytes: int = 0, stream=None):
+    """Like ``dasc_restore`` with the dequantisation fused in; ``pool`` is a byte (uint8) tensor."""
+    _check(lib().dasc_restore_int8(plan.handle, _ptr(pool), slot_stride_bytes, _ptr(src_slot), _ptr(state),
+                                   layer_stride, req_stride, _ptr(dst_req), int(src_slot.numel()),
+                                   _stream_ptr(stream)), "dasc_restore_int8")
 
 
 def dasc_refresh_workspace_bytes(plan: Plan, n_req: int, n_layers_in_call: int, algo: int = ALGO_AUTO) -> int:

@@ -156,6 +156,52 @@ dasc_status_t dasc_restore(const dasc_plan_t *plan, const float *pool_base, int6
   return e == 0 ? DASC_OK : DASC_ERR_CUDA;
 }
 
+static int64_t int8_slot_bytes(const dasc_plan_t *plan) {
+  const int64_t raw = plan->packed_rows * (plan->info.d_v + 4);
+  return (raw + 15) / 16 * 16;
+}
+
+static dasc_status_t check_int8_args(const dasc_plan_t *plan, const void *state, int64_t layer_stride,
+                                     int64_t req_stride, const void *idx_a, const void *pool,
+                                     int64_t *slot_stride_bytes, const void *idx_b, int32_t n_pairs) {
+  int64_t fp32_stride = 0;  // the fp32 slot rule does not apply; everything else does
+  dasc_status_t st = check_copy_args(plan, state, layer_stride, req_stride, idx_a, pool, &fp32_stride, idx_b, n_pairs);
+  if (st != DASC_OK || n_pairs == 0) return st;
+  const int64_t d_v = plan->info.d_v;
+  if (d_v < 4 || d_v > 128 || (d_v & (d_v - 1))) return DASC_ERR_SHAPE;
+  if (*slot_stride_bytes == 0) *slot_stride_bytes = int8_slot_bytes(plan);
+  if (*slot_stride_bytes < int8_slot_bytes(plan) || *slot_stride_bytes % 16) return DASC_ERR_INVALID_ARG;
+  return DASC_OK;
+}
+
+dasc_status_t dasc_int8_slot_bytes(const dasc_plan_t *plan, size_t *out) {
+  if (!plan || !out) return DASC_ERR_INVALID_ARG;
+  *out = static_cast<size_t>(int8_slot_bytes(plan));
+  return DASC_OK;
+}
+
+dasc_status_t dasc_pack_int8(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride,
+                             int64_t req_stride, const int32_t *src_req, void *pool_base, int64_t slot_stride_bytes,
+                             const int32_t *dst_slot, int32_t n_pairs, void *cuda_stream) {
+  dasc_status_t st = check_int8_args(plan, state_base, layer_stride, req_stride, src_req, pool_base,
+                                     &slot_stride_bytes, dst_slot, n_pairs);
+  if (st != DASC_OK || n_pairs == 0) return st;
+  const int e = dasc_launch_pack_int8(plan, state_base, layer_stride, req_stride, src_req, pool_base,
+                                      slot_stride_bytes, dst_slot, n_pairs, cuda_stream);
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+dasc_status_t dasc_restore_int8(const dasc_plan_t *plan, const void *pool_base, int64_t slot_stride_bytes,
+                                const int32_t *src_slot, float *state_base, int64_t layer_stride, int64_t req_stride,
+                                const int32_t *dst_req, int32_t n_pairs, void *cuda_stream) {
+  dasc_status_t st = check_int8_args(plan, state_base, layer_stride, req_stride, dst_req, pool_base,
+                                     &slot_stride_bytes, src_slot, n_pairs);
+  if (st != DASC_OK || n_pairs == 0) return st;
+  const int e = dasc_launch_restore_int8(plan, pool_base, slot_stride_bytes, src_slot, state_base, layer_stride,
+                                         req_stride, dst_req, n_pairs, cuda_stream);
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
 static bool chunked_shape_ok(const dasc_plan_t *plan) { return plan->info.d_k == 128 && plan->info.d_v == 128; }
 
 dasc_status_t dasc_refresh_workspace_bytes(const dasc_plan_t *plan, int32_t n_req, int32_t n_layers_in_call,

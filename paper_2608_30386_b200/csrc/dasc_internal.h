@@ -42,6 +42,14 @@ int dasc_launch_restore(const dasc_plan_s *plan, const float *pool, int64_t slot
                         float *state, int64_t layer_stride, int64_t req_stride, const int32_t *dst_req,
                         int32_t n_pairs, void *stream);
 
+// codec_int8.cu
+int dasc_launch_pack_int8(const dasc_plan_s *plan, const float *state, int64_t layer_stride, int64_t req_stride,
+                          const int32_t *src_req, void *pool, int64_t slot_stride_bytes, const int32_t *dst_slot,
+                          int32_t n_pairs, void *stream);
+int dasc_launch_restore_int8(const dasc_plan_s *plan, const void *pool, int64_t slot_stride_bytes,
+                             const int32_t *src_slot, float *state, int64_t layer_stride, int64_t req_stride,
+                             const int32_t *dst_req, int32_t n_pairs, void *stream);
+
 struct DascRefreshArgs {
   int32_t kind, H_v, H_k, d_k, d_v;
   float *state;
