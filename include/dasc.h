@@ -7,6 +7,8 @@
  *   dasc_pack     device retained units -> ragged pool  (Store path, Section 4.1, App. B Scheme 2)
  *   dasc_restore  device pool -> dense state, zero-fill (Load path, zero-fill policy, Section 4.2)
  *   dasc_refresh  device replay of the gated delta rule (Eq. 1; suffix-refresh policy, Section 4.2)
+ *   dasc_pack_int8 / dasc_restore_int8
+ *                 device the same copies with the INT8 checkpoint codec fused in (Appendix D, Eq. 10)
  *
  * Conventions
  *   - No exception crosses this boundary; every call returns a dasc_status_t.

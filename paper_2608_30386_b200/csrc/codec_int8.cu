@@ -15,13 +15,19 @@
 namespace {
 
 #ifndef DASC_INT8_THREADS
-#define DASC_INT8_THREADS 256
+#define DASC_INT8_THREADS 128
 #endif
 #ifndef DASC_INT8_PACK_UNROLL
 #define DASC_INT8_PACK_UNROLL 4
 #endif
 #ifndef DASC_INT8_RESTORE_UNROLL
 #define DASC_INT8_RESTORE_UNROLL 4
+#endif
+#ifndef DASC_INT8_PACK_MIN_BLOCKS
+#define DASC_INT8_PACK_MIN_BLOCKS 12   /* caps registers at 40: occupancy is what hides the latency */
+#endif
+#ifndef DASC_INT8_RESTORE_MIN_BLOCKS
+#define DASC_INT8_RESTORE_MIN_BLOCKS 16   /* caps registers at 32 */
 #endif
 constexpr int kThreads = DASC_INT8_THREADS;          // tuning knobs; defaults = best of a measured sweep
 constexpr int kUnroll = DASC_INT8_PACK_UNROLL;       // rows (pack) / vectors (restore) in flight per thread
@@ -68,19 +74,31 @@ constexpr float kSafeFraction = 0.5f - 1.0f / 8192.0f;
 // |x / s| < 127.5.)
 __device__ __forceinline__ uint32_t codes_of(const uint4 &v, float a) {
   float inv;  // the argument lies in [7.8e-11, 2.7e36], so the reciprocal is a normal number
-  asm("rcp.approx.f32 %0, %1;" : "=f"(inv) : "f"(__fmul_rn(fmaxf(a, 1e-8f), 1.0f / 127.0f)));
-  const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(__fmul_rn(fmaxf(a, 1e-8f), 1.0f / 127.0f)));
+  // two values per instruction (packed fp32 pairs): m = x*inv + magic (one rounding: the nearest
+  // integer of the product), r = m - magic, d = x*inv - r = signed distance of the product to it
   uint32_t m[4];
-  float worst = 0.0f;
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const float t = __fmul_rn(__uint_as_float(in[e]), inv);
-    const float r = __fadd_rn(t, kRoundMagic);
-    m[e] = __float_as_uint(r);
-    worst = fmaxf(worst, fabsf(__fsub_rn(t, __fsub_rn(r, kRoundMagic))));
-  }
+  float d[4];
+  asm("{\n\t.reg .b64 xa, xb, iv, mg, ma, mb, ra, rb;\n\t"
+      "mov.b64 xa, {%8, %9};\n\t"
+      "mov.b64 xb, {%10, %11};\n\t"
+      "mov.b64 iv, {%12, %12};\n\t"
+      "mov.b64 mg, {%13, %13};\n\t"
+      "fma.rn.f32x2 ma, xa, iv, mg;\n\t"
+      "fma.rn.f32x2 mb, xb, iv, mg;\n\t"
+      "sub.rn.f32x2 ra, mg, ma;\n\t"  // -(r)
+      "sub.rn.f32x2 rb, mg, mb;\n\t"
+      "fma.rn.f32x2 ra, xa, iv, ra;\n\t"
+      "fma.rn.f32x2 rb, xb, iv, rb;\n\t"
+      "mov.b64 {%0, %1}, ma;\n\t"
+      "mov.b64 {%2, %3}, mb;\n\t"
+      "mov.b64 {%4, %5}, ra;\n\t"
+      "mov.b64 {%6, %7}, rb;\n\t}"
+      : "=r"(m[0]), "=r"(m[1]), "=r"(m[2]), "=r"(m[3]), "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "f"(inv), "f"(kRoundMagic));
+  const float worst = fmaxf(fmaxf(fabsf(d[0]), fabsf(d[1])), fmaxf(fabsf(d[2]), fabsf(d[3])));
   uint32_t word = __byte_perm(__byte_perm(m[0], m[1], 0x0040), __byte_perm(m[2], m[3], 0x0040), 0x5410);
-  if (!(worst < kSafeFraction)) {  // rare; also catches non-finite intermediates
+  if (!(worst < kSafeFraction)) {  // rare
     const float s = __fdiv_rn(fmaxf(a, 1e-8f), 127.0f);
     word = code_exact(v.x, s) | (code_exact(v.y, s) << 8) | (code_exact(v.z, s) << 16) | (code_exact(v.w, s) << 24);
   }
@@ -96,7 +114,7 @@ __device__ __forceinline__ float absmax4(const uint4 &v) {
 // a row is held by `lanes_per_row` = d_v/4 consecutive lanes of one warp (a power of two <= 32).
 // FULL_WARP_ROWS: d_v = 128, a row is exactly one warp and the abs-max is one warp reduction.
 template <bool FULL_WARP_ROWS>
-__global__ void __launch_bounds__(kThreads) pack_int8_kernel(const uint4 *__restrict__ state, int64_t layer_stride4,
+__global__ void __launch_bounds__(kThreads, DASC_INT8_PACK_MIN_BLOCKS) pack_int8_kernel(const uint4 *__restrict__ state, int64_t layer_stride4,
                                                              int64_t req_stride4, const int32_t *__restrict__ src_req,
                                                              uint8_t *__restrict__ pool, int64_t slot_stride_bytes,
                                                              const int32_t *__restrict__ dst_slot,
@@ -163,21 +181,40 @@ __global__ void __launch_bounds__(kThreads) pack_int8_kernel(const uint4 *__rest
   }
 }
 
-// S_hat = q * s.  q is rebuilt without an integer-to-float conversion: byte b = q + 128 placed in the
-// low mantissa bits of 2^23 gives 2^23 + b exactly, and subtracting 2^23 + 128 leaves q.
-__device__ __forceinline__ float dequant(uint32_t biased_word, uint32_t selector, float s) {
-  const float f = __uint_as_float(__byte_perm(biased_word, 0x4B000000u, selector));
-  return __fmul_rn(__fsub_rn(f, 8388736.0f), s);
+// S_hat = q * s for the four codes of one word.  q is rebuilt without an integer-to-float
+// conversion: byte b = q + 128 placed in the low mantissa bits of 2^23 gives 2^23 + b exactly, and
+// subtracting 2^23 + 128 leaves q; then one fp32 multiply, two values per instruction.
+__device__ __forceinline__ uint4 dequant4(uint32_t word, float s) {
+  const uint32_t w = word ^ 0x80808080u;
+  uint4 out;
+  asm("{\n\t.reg .b64 fa, fb, of, sc;\n\t"
+      "mov.b64 fa, {%4, %5};\n\t"
+      "mov.b64 fb, {%6, %7};\n\t"
+      "mov.b64 of, {%8, %8};\n\t"
+      "mov.b64 sc, {%9, %9};\n\t"
+      "sub.rn.f32x2 fa, fa, of;\n\t"
+      "sub.rn.f32x2 fb, fb, of;\n\t"
+      "mul.rn.f32x2 fa, fa, sc;\n\t"
+      "mul.rn.f32x2 fb, fb, sc;\n\t"
+      "mov.b64 {%0, %1}, fa;\n\t"
+      "mov.b64 {%2, %3}, fb;\n\t}"
+      : "=r"(out.x), "=r"(out.y), "=r"(out.z), "=r"(out.w)
+      : "r"(__byte_perm(w, 0x4B000000u, 0x7540)), "r"(__byte_perm(w, 0x4B000000u, 0x7541)),
+        "r"(__byte_perm(w, 0x4B000000u, 0x7542)), "r"(__byte_perm(w, 0x4B000000u, 0x7543)), "f"(8388736.0f), "f"(s));
+  return out;
 }
+
 // grid = (ceil(layer_vecs / (kThreads*kRUnroll)), n_layers, pairs).
-__global__ void __launch_bounds__(kThreads) restore_int8_kernel(const uint8_t *__restrict__ pool,
+template <bool FULL_WARP_ROWS>
+__global__ void __launch_bounds__(kThreads, DASC_INT8_RESTORE_MIN_BLOCKS) restore_int8_kernel(const uint8_t *__restrict__ pool,
                                                                 int64_t slot_stride_bytes,
                                                                 const int32_t *__restrict__ src_slot,
                                                                 uint4 *__restrict__ state, int64_t layer_stride4,
                                                                 int64_t req_stride4, const int32_t *__restrict__ dst_req,
                                                                 const int32_t *__restrict__ row_pos, uint32_t layer_vecs,
                                                                 uint32_t rows_per_layer, uint32_t packed_rows,
-                                                                uint32_t lanes_per_row, int32_t n_pairs) {
+                                                                uint32_t lanes_per_row_arg, int32_t n_pairs) {
+  const uint32_t lanes_per_row = FULL_WARP_ROWS ? 32u : lanes_per_row_arg;
   const uint32_t base = blockIdx.x * (kThreads * kRUnroll) + threadIdx.x;
   const int32_t layer = blockIdx.y;
   const int32_t *pos_l = row_pos + static_cast<int64_t>(layer) * rows_per_layer;
@@ -187,21 +224,18 @@ __global__ void __launch_bounds__(kThreads) restore_int8_kernel(const uint8_t *_
     const float *scales = reinterpret_cast<const float *>(slot + static_cast<size_t>(packed_rows) * lanes_per_row * 4u);
     uint4 *dst_base = state + static_cast<int64_t>(__ldg(dst_req + pair)) * req_stride4 + layer * layer_stride4;
     uint32_t word[kRUnroll];
-    float scale[kRUnroll];
-    bool keep[kRUnroll];
+    float scale[kRUnroll];  // 0 marks an omitted row: a stored scale is at least 1e-8/127
 #pragma unroll
     for (int u = 0; u < kRUnroll; ++u) {
       const uint32_t i = base + u * kThreads;
       word[u] = 0u;
       scale[u] = 0.0f;
-      keep[u] = false;
       if (i < layer_vecs) {
         const uint32_t row = i / lanes_per_row;
         const uint32_t vec = i - row * lanes_per_row;
         const int32_t pos = __ldg(pos_l + row);
         if (pos >= 0) {
-          keep[u] = true;
-          word[u] = ld_stream32(codes + static_cast<int64_t>(pos) * lanes_per_row + vec);
+          word[u] = ld_stream32(codes + static_cast<uint32_t>(pos) * lanes_per_row + vec);
           scale[u] = __ldg(scales + pos);
         }
       }
@@ -209,17 +243,8 @@ __global__ void __launch_bounds__(kThreads) restore_int8_kernel(const uint8_t *_
 #pragma unroll
     for (int u = 0; u < kRUnroll; ++u) {
       const uint32_t i = base + u * kThreads;
-      if (i < layer_vecs) {
-        uint4 out = make_uint4(0u, 0u, 0u, 0u);  // omitted rows: +0.0f
-        if (keep[u]) {
-          const uint32_t w = word[u] ^ 0x80808080u;
-          out.x = __float_as_uint(dequant(w, 0x7540, scale[u]));
-          out.y = __float_as_uint(dequant(w, 0x7541, scale[u]));
-          out.z = __float_as_uint(dequant(w, 0x7542, scale[u]));
-          out.w = __float_as_uint(dequant(w, 0x7543, scale[u]));
-        }
-        st_stream(dst_base + i, out);
-      }
+      // an omitted row has all codes 0 and scale 0: 0 * 0 = +0.0f, the zero fill
+      if (i < layer_vecs) st_stream(dst_base + i, dequant4(word[u], scale[u]));
     }
   }
 }
@@ -252,7 +277,8 @@ int dasc_launch_restore_int8(const dasc_plan_s *plan, const void *pool, int64_t 
   const uint32_t per_block = kThreads * kRUnroll;
   dim3 grid(static_cast<uint32_t>((layer_vecs + per_block - 1) / per_block),
             static_cast<uint32_t>(plan->info.n_layers), static_cast<uint32_t>(n_pairs < 65535 ? n_pairs : 65535));
-  restore_int8_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+  auto kernel = lpr == 32 ? restore_int8_kernel<true> : restore_int8_kernel<false>;
+  kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const uint8_t *>(pool), slot_stride_bytes, src_slot, reinterpret_cast<uint4 *>(state),
       layer_stride / 4, req_stride / 4, dst_req, plan->d_row_pos, static_cast<uint32_t>(layer_vecs),
       static_cast<uint32_t>(plan->rows_per_layer), static_cast<uint32_t>(plan->packed_rows), lpr, n_pairs);
