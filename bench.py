@@ -369,6 +369,31 @@ def main():
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
     t_pack, t_restore, t_refresh, t_total = times.tolist()
 
+    # ---- the paper's own load policy (Section 4.2): replay the last W tokens from a zero scratch state, merge the
+    #      omitted units, no outputs (state-only fast path).  Same streams, W = the suffix length. ----
+    wb = torch.empty(N_REQ, dtype=torch.int32, device=dev)
+
+    def window_step():
+        for gi in range(n_groups):
+            dasc.dasc_refresh_window(plan, active, layer_stride, req_stride, ids, None, k, v, g, beta, cu, T, wb,
+                                     window=SUFFIX, layer_begin=gi * group, layer_end=(gi + 1) * group, algo=algo,
+                                     workspace=ws)
+
+    for _ in range(3):
+        window_step()
+    barrier()
+    ev_w = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ev_w[0].record(stream)
+    for _ in range(args.steps):
+        window_step()
+    ev_w[1].record(stream)
+    barrier()
+    assert dasc.dasc_refresh_status(ws) == 0
+    t_window = torch.tensor([ev_w[0].elapsed_time(ev_w[1]) / args.steps], dtype=torch.float64, device=dev)
+    if dist:
+        dist.all_reduce(t_window, op=dist.ReduceOp.MAX)
+    t_window = float(t_window)
+
     # ---- end-to-end leg: host buffers, copies inside the timed region -------------------------
     e2e = None
     if not args.no_e2e:
@@ -481,6 +506,9 @@ def main():
         "pack_GBps": world * pack_gbs, "restore_GBps": world * restore_gbs,
         "refresh_tokens_per_s": world * N_REQ * SUFFIX / (t_refresh * 1e-3),
         "refresh_token_heads_per_s": world * token_heads / (t_refresh * 1e-3),
+        # dasc_refresh_window: scratch replay of the last `suffix_tokens` tokens, merge of omitted units, no outputs
+        "window_refresh_state_only": {"ms": t_window, "tokens_per_s": world * N_REQ * SUFFIX / (t_window * 1e-3),
+                                      "token_heads_per_s": world * token_heads / (t_window * 1e-3)},
         "roofline": roofline, "roofline_by_kernel": rl, "clocks": clocks,
         "gpu_launches": (2 + n_groups) * args.steps,
     }

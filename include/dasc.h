@@ -274,6 +274,39 @@ dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t l
 dasc_status_t dasc_refresh_status(const void *workspace, size_t workspace_bytes);
 
 /*
+ * Load path, suffix-refresh policy as the paper states it (Section 4.2, with the
+ * window of Eq. 7): after dasc_restore has loaded the retained units of a hit,
+ * each request's last `window` tokens BEFORE the cache boundary are replayed
+ * from a zero scratch state, and only the units the plan omits are copied from
+ * the scratch state into the stored state (SCRATCH_MERGE_LOCAL); retained units
+ * keep their exactly loaded values.  A request whose available prefix is
+ * shorter than the window replays the whole prefix (Table 8: replayed tokens
+ * per hit are the window clipped by the prefix).
+ *   cu_seqlens   DEVICE int32[n_req+1]: request r's available prefix is tokens
+ *                [cu_seqlens[r], cu_seqlens[r+1]) of the streams; the replayed
+ *                range is [max(cu_seqlens[r], cu_seqlens[r+1] - window), cu_seqlens[r+1]).
+ *   window       W_replay in tokens; <= 0 means the plan's own W_replay (Eq. 7).
+ *                When that is 0 (nothing omitted) only window_begin is written.
+ *   window_begin DEVICE int32[n_req], written by the call: first replayed token
+ *                of each request (cu_seqlens[r+1] - window_begin[r] tokens are
+ *                replayed); caller-owned, must stay valid until the call completes.
+ *   q, o         outputs are not part of this policy: pass o = NULL, and then q
+ *                may be NULL too and the kernels skip the output side entirely
+ *                (state-only fast path).  With o != NULL outputs of the replayed
+ *                tokens are written at their stream positions (from the scratch
+ *                state, i.e. without the retained history).
+ * Everything else as for dasc_refresh (mode is fixed; max_seqlen is the window).
+ */
+dasc_status_t dasc_refresh_window(const dasc_plan_t *plan, float *state_base, int64_t layer_stride,
+                                  int64_t req_stride, const int32_t *req_idx, const void *q,
+                                  const void *k, const void *v, int32_t io_dtype, const float *g,
+                                  const float *beta, const int32_t *cu_seqlens, int32_t n_req,
+                                  int64_t total_tokens, int64_t window, int32_t layer_begin,
+                                  int32_t layer_end, float q_scale, void *o, int32_t o_dtype,
+                                  int32_t algo, int32_t *window_begin, void *workspace,
+                                  size_t workspace_bytes, void *cuda_stream);
+
+/*
  * The paper has no counterpart to this call: it is dasc_refresh (chunked tensor-core kernel,
  * bf16 token streams, d_k = d_v = 128) for callers that cannot hand over a workspace because
  * they cannot allocate device memory at the point of the call.  The typical case is a serving

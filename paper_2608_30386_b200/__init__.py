@@ -7,6 +7,6 @@ declared in ``include/dasc.h``); this package only marshals arguments.
 from .binding import (  # noqa: F401
     ALGO_AUTO, ALGO_CHUNKED, ALGO_SEQUENTIAL, GDN, IO_BF16, IO_FP32, KDA, REFRESH_CONTINUE,
     REFRESH_SCRATCH_MERGE_LOCAL, SCOPE_HEAD, SCOPE_LAYER, SCOPE_MODEL, SEL_EXPLICIT, SEL_THRESHOLD, SEL_TOP_RATIO,
-    DascError, Plan, dasc_pack, dasc_plan, dasc_refresh, dasc_refresh_static, dasc_refresh_status, dasc_refresh_workspace_bytes,
+    DascError, Plan, dasc_pack, dasc_plan, dasc_refresh, dasc_refresh_static, dasc_refresh_status, dasc_refresh_window, dasc_refresh_workspace_bytes,
     dasc_int8_slot_bytes, dasc_pack_int8, dasc_restore, dasc_restore_int8, lib, status_string, version,
 )

@@ -30,7 +30,7 @@ EXPORTS = (
     "dasc_plan", "dasc_plan_destroy", "dasc_plan_info", "dasc_plan_horizon", "dasc_plan_mask",
     "dasc_plan_window", "dasc_plan_layer_counts", "dasc_plan_layer_offsets", "dasc_pack", "dasc_restore",
     "dasc_int8_slot_bytes", "dasc_pack_int8", "dasc_restore_int8",
-    "dasc_refresh_workspace_bytes", "dasc_refresh", "dasc_refresh_status", "dasc_refresh_static",
+    "dasc_refresh_workspace_bytes", "dasc_refresh", "dasc_refresh_status", "dasc_refresh_window", "dasc_refresh_static",
     "dasc_status_string", "dasc_version",
 )
 
@@ -99,6 +99,10 @@ def lib() -> C.CDLL:
                                    C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]
         L.dasc_refresh_status.argtypes = [C.c_void_p, C.c_size_t]
+        L.dasc_refresh_window.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
+                                          C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.dasc_refresh_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                           C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
@@ -268,6 +272,27 @@ def dasc_refresh(plan: Plan, state: torch.Tensor, layer_stride: int, req_stride:
                               _ptr(v), io, _ptr(g), _ptr(beta), _ptr(cu_seqlens), int(cu_seqlens.numel() - 1),
                               int(total_tokens), int(max_seqlen), layer_begin, layer_end, float(q_scale), _ptr(o),
                               o_io, mode, algo, _ptr(workspace), ws_bytes, _stream_ptr(stream)), "dasc_refresh")
+
+
+def dasc_refresh_window(plan: Plan, state: torch.Tensor, layer_stride: int, req_stride: int, req_idx: torch.Tensor,
+                        q: torch.Tensor | None, k: torch.Tensor, v: torch.Tensor, g: torch.Tensor, beta: torch.Tensor,
+                        cu_seqlens: torch.Tensor, total_tokens: int, window_begin: torch.Tensor, *, window: int = 0,
+                        layer_begin: int = 0, layer_end: int | None = None, q_scale: float = 1.0,
+                        o: torch.Tensor | None = None, algo: int = ALGO_AUTO, workspace: torch.Tensor | None = None,
+                        stream=None):
+    """The paper's suffix-refresh load policy: replay each request's last ``window`` prefix tokens (0 = the
+    plan's W_replay) from a zero scratch state and merge only the omitted units.  ``window_begin`` (int32
+    [n_req], device) receives the first replayed token of each request.  ``q`` may be None when ``o`` is."""
+    io = IO_BF16 if k.dtype == torch.bfloat16 else IO_FP32
+    o_io = IO_BF16 if (o is not None and o.dtype == torch.bfloat16) else IO_FP32
+    if layer_end is None:
+        layer_end = plan.info.n_layers
+    ws_bytes = int(workspace.numel() * workspace.element_size()) if workspace is not None else 0
+    _check(lib().dasc_refresh_window(plan.handle, _ptr(state), layer_stride, req_stride, _ptr(req_idx), _ptr(q),
+                                     _ptr(k), _ptr(v), io, _ptr(g), _ptr(beta), _ptr(cu_seqlens),
+                                     int(cu_seqlens.numel() - 1), int(total_tokens), int(window), layer_begin,
+                                     layer_end, float(q_scale), _ptr(o), o_io, algo, _ptr(window_begin),
+                                     _ptr(workspace), ws_bytes, _stream_ptr(stream)), "dasc_refresh_window")
 
 
 def dasc_refresh_status(workspace: torch.Tensor | None) -> int:

@@ -66,6 +66,17 @@ dasc_status_t check_copy_args(const dasc_plan_t *plan, const void *state, int64_
   return DASC_OK;
 }
 
+// first replayed token of each request: max(cu[r], cu[r+1] - window)
+__global__ void window_begin_kernel(const int32_t *__restrict__ cu, int32_t n_req, int64_t window,
+                                    int32_t *__restrict__ out) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r < n_req) {
+    const int64_t lo = cu[r], hi = cu[r + 1];
+    const int64_t b = hi - window;
+    out[r] = static_cast<int32_t>(b > lo ? b : lo);
+  }
+}
+
 }  // namespace
 
 extern "C" {
@@ -213,13 +224,16 @@ dasc_status_t dasc_refresh_workspace_bytes(const dasc_plan_t *plan, int32_t n_re
   return DASC_OK;
 }
 
-dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t layer_stride, int64_t req_stride,
-                           const int32_t *req_idx, const void *q, const void *k, const void *v, int32_t io_dtype,
-                           const float *g, const float *beta, const int32_t *cu_seqlens, int32_t n_req,
-                           int64_t total_tokens, int32_t max_seqlen, int32_t layer_begin, int32_t layer_end,
-                           float q_scale, void *o, int32_t o_dtype, int32_t mode, int32_t algo, void *workspace,
-                           size_t workspace_bytes, void *cuda_stream) {
+// tok_begin: device array of first tokens (null = cu_seqlens[r]).  q may be null when o is null.
+static dasc_status_t refresh_impl(const dasc_plan_t *plan, float *state_base, int64_t layer_stride, int64_t req_stride,
+                                  const int32_t *req_idx, const void *q, const void *k, const void *v,
+                                  int32_t io_dtype, const float *g, const float *beta, const int32_t *cu_seqlens,
+                                  const int32_t *tok_begin, int32_t n_req, int64_t total_tokens, int32_t max_seqlen,
+                                  int32_t layer_begin, int32_t layer_end, float q_scale, void *o, int32_t o_dtype,
+                                  int32_t mode, int32_t algo, void *workspace, size_t workspace_bytes,
+                                  void *cuda_stream) {
   if (!plan || plan->info.device < 0) return DASC_ERR_INVALID_ARG;
+  if (!q && !o) q = k;  // never read for its values: the kernels skip or discard the output side
   if (n_req < 0 || total_tokens < 0 || max_seqlen < 0) return DASC_ERR_INVALID_ARG;
   if (layer_begin < 0 || layer_end < layer_begin || layer_end > plan->info.n_layers) return DASC_ERR_INVALID_ARG;
   if (io_dtype != DASC_IO_BF16 && io_dtype != DASC_IO_FP32) return DASC_ERR_INVALID_ARG;
@@ -257,6 +271,7 @@ dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t l
   a.g = g;
   a.beta = beta;
   a.cu_seqlens = cu_seqlens;
+  a.tok_begin = tok_begin;
   a.n_req = n_req;
   a.total_tokens = total_tokens;
   a.max_seqlen = max_seqlen;
@@ -286,6 +301,40 @@ dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t l
   }
   if (e == -1) return DASC_ERR_SHAPE;
   return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t layer_stride, int64_t req_stride,
+                           const int32_t *req_idx, const void *q, const void *k, const void *v, int32_t io_dtype,
+                           const float *g, const float *beta, const int32_t *cu_seqlens, int32_t n_req,
+                           int64_t total_tokens, int32_t max_seqlen, int32_t layer_begin, int32_t layer_end,
+                           float q_scale, void *o, int32_t o_dtype, int32_t mode, int32_t algo, void *workspace,
+                           size_t workspace_bytes, void *cuda_stream) {
+  if (!q) return n_req == 0 || total_tokens == 0 || layer_end == layer_begin ? DASC_OK : DASC_ERR_INVALID_ARG;
+  return refresh_impl(plan, state_base, layer_stride, req_stride, req_idx, q, k, v, io_dtype, g, beta, cu_seqlens,
+                      nullptr, n_req, total_tokens, max_seqlen, layer_begin, layer_end, q_scale, o, o_dtype, mode, algo,
+                      workspace, workspace_bytes, cuda_stream);
+}
+
+dasc_status_t dasc_refresh_window(const dasc_plan_t *plan, float *state_base, int64_t layer_stride,
+                                  int64_t req_stride, const int32_t *req_idx, const void *q, const void *k,
+                                  const void *v, int32_t io_dtype, const float *g, const float *beta,
+                                  const int32_t *cu_seqlens, int32_t n_req, int64_t total_tokens, int64_t window,
+                                  int32_t layer_begin, int32_t layer_end, float q_scale, void *o, int32_t o_dtype,
+                                  int32_t algo, int32_t *window_begin, void *workspace, size_t workspace_bytes,
+                                  void *cuda_stream) {
+  if (!plan || plan->info.device < 0 || n_req < 0) return DASC_ERR_INVALID_ARG;
+  if (o && !q) return DASC_ERR_INVALID_ARG;
+  if (window <= 0) window = plan->info.w_replay;
+  if (n_req == 0) return DASC_OK;
+  if (!cu_seqlens || !window_begin) return DASC_ERR_INVALID_ARG;
+  if (window > INT32_MAX) window = INT32_MAX;
+  window_begin_kernel<<<(n_req + 255) / 256, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(cu_seqlens, n_req, window,
+                                                                                               window_begin);
+  if (cudaGetLastError() != cudaSuccess) return DASC_ERR_CUDA;
+  if (window == 0) return DASC_OK;  // nothing is omitted, so nothing needs a refresh
+  return refresh_impl(plan, state_base, layer_stride, req_stride, req_idx, q, k, v, io_dtype, g, beta, cu_seqlens,
+                      window_begin, n_req, total_tokens, static_cast<int32_t>(window), layer_begin, layer_end, q_scale,
+                      o, o_dtype, DASC_REFRESH_SCRATCH_MERGE_LOCAL, algo, workspace, workspace_bytes, cuda_stream);
 }
 
 dasc_status_t dasc_refresh_status(const void *workspace, size_t workspace_bytes) {

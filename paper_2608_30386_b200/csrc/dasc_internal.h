@@ -59,6 +59,7 @@ struct DascRefreshArgs {
   int32_t io_bf16;
   const float *g, *beta;
   const int32_t *cu_seqlens;
+  const int32_t *tok_begin;  // device, [n_req], or null: first token of each request (null = cu_seqlens[r])
   int32_t n_req;
   int64_t total_tokens;
   int32_t max_seqlen;

@@ -163,7 +163,9 @@ __device__ __forceinline__ void warp_mm_store(float *Cb, const float (&acc)[2][4
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-template <bool KDA, typename OT>
+// WITH_O = false is the state-only variant (no outputs wanted): q is never read, the Qt rows, P and the
+// output product are left out.
+template <bool KDA, typename OT, bool WITH_O>
 __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs a) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t{1023});
@@ -184,7 +186,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   const int r = blockIdx.x / (a.H_v * a.n_layers_in_call);
   const int hk = h / (a.H_v / a.H_k);
   const int layer = a.layer_begin + lc;
-  const int64_t t_begin = a.cu_seqlens[r];
+  const int64_t t_begin = a.tok_begin ? a.tok_begin[r] : a.cu_seqlens[r];
   const int n_tok = static_cast<int>(a.cu_seqlens[r + 1] - t_begin);
   if (n_tok <= 0 && a.mode == DASC_REFRESH_CONTINUE) return;
 
@@ -196,7 +198,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   const __nv_bfloat16 *gv = static_cast<const __nv_bfloat16 *>(a.v) + (tok0 * a.H_v + h) * D;
   const float *gg = a.g + (tok0 * a.H_v + h) * (KDA ? D : 1);
   const float *gb = a.beta + tok0 * a.H_v + h;
-  OT *go = a.o ? static_cast<OT *>(a.o) + (tok0 * a.H_v + h) * D : nullptr;
+  OT *const go = WITH_O ? static_cast<OT *>(a.o) + (tok0 * a.H_v + h) * D : nullptr;
   const int64_t qk_stride = static_cast<int64_t>(a.H_k) * D, v_stride = static_cast<int64_t>(a.H_v) * D;
   const int64_t g_stride = static_cast<int64_t>(a.H_v) * (KDA ? D : 1), b_stride = a.H_v;
 
@@ -252,7 +254,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 #pragma unroll 1
         for (int kk = 0; kk < 16; ++kk)
           mma_ts(tm + COL_RO, tm + COL_S + kk * 8, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
-                 ID_N64, kk != 0);
+                 go ? ID_N64 : ID_N32, kk != 0);  // without outputs only the Kt rows are needed
         mma_commit(&misc->bar_ro);
       }
       // MMA3: U^T = RHS^T T^T; RHS^T is a tf32 pair (high part over R^T, low part in the A|P columns)
@@ -300,7 +302,8 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         const int t = i >> 4, j = i & 15;
         const bool valid = t < ntok;
         const int64_t tt = t0 + (valid ? t : 0);
-        cp_async16_zfill(sbase + OFF_RAWQ + t * 256 + j * 16, reinterpret_cast<const char *>(gq + tt * qk_stride) + j * 16, valid);
+        if (go)  // no outputs wanted: q is never read
+          cp_async16_zfill(sbase + OFF_RAWQ + t * 256 + j * 16, reinterpret_cast<const char *>(gq + tt * qk_stride) + j * 16, valid);
         cp_async16_zfill(sbase + OFF_RAWK + t * 256 + j * 16, reinterpret_cast<const char *>(gk + tt * qk_stride) + j * 16, valid);
       }
     };
@@ -388,7 +391,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           kraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWK + (t4 + j) * 256 + c0 * 2);
-          qraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + (t4 + j) * 256 + c0 * 2);
+          qraw[j] = go ? *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + (t4 + j) * 256 + c0 * 2) : make_uint2(0u, 0u);
           if constexpr (KDA) {
             const float4 g4 = *reinterpret_cast<const float4 *>(smem + OFF_G + (t4 + j) * 512 + c0 * 4);
             gl[j][0] = g4.x; gl[j][1] = g4.y; gl[j][2] = g4.z; gl[j][3] = g4.w;
@@ -439,7 +442,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
             kht[i][j] = kh[i];
           }
           *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, t, c0)) = make_uint4(kt[0], kt[1], kt[2], kt[3]);
-          *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, 32 + t, c0)) = make_uint4(qt[0], qt[1], qt[2], qt[3]);
+          if (go) *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, 32 + t, c0)) = make_uint4(qt[0], qt[1], qt[2], qt[3]);
           *reinterpret_cast<uint4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_uint4(kh[0], kh[1], kh[2], kh[3]);
         }
 #pragma unroll
@@ -534,7 +537,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
             warp_mm_acc(acc2, Xm + 16 * LDX + 16, Xm + 16, lane);
             warp_mm_store(Xm + 16 * LDX, acc2, -1.f, lane);
           }
-        } else {
+        } else if (go) {
           // lanes 32-63: row t of P = lower_incl_diag(Qt Kh^T), straight to its operand tile
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
@@ -683,9 +686,9 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   if (warp == 8) tmem_dealloc(tm, TMEM_COLS);
 }
 
-template <bool KDA, typename OT>
+template <bool KDA, typename OT, bool WITH_O>
 int launch(const DascRefreshArgs &a, void *stream) {
-  auto kern = refresh_chunked_kernel<KDA, OT>;
+  auto kern = refresh_chunked_kernel<KDA, OT, WITH_O>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SMEM_ALLOC));
   if (e != cudaSuccess) return static_cast<int>(e);
   const int64_t n_units = static_cast<int64_t>(a.n_req) * a.n_layers_in_call * a.H_v;
@@ -707,9 +710,9 @@ size_t dasc_refresh_chunked_workspace_bytes(int32_t, int32_t, int32_t) { return 
 int dasc_launch_refresh_chunked(const DascRefreshArgs &a, void *stream) {
   if (a.d_k != D || a.d_v != D || !a.io_bf16) return -1;
   const bool kda = a.kind == DASC_KDA;
-  const bool o_bf16 = a.o ? a.o_bf16 != 0 : true;
-  if (o_bf16) return kda ? launch<true, __nv_bfloat16>(a, stream) : launch<false, __nv_bfloat16>(a, stream);
-  return kda ? launch<true, float>(a, stream) : launch<false, float>(a, stream);
+  if (!a.o) return kda ? launch<true, __nv_bfloat16, false>(a, stream) : launch<false, __nv_bfloat16, false>(a, stream);
+  if (a.o_bf16) return kda ? launch<true, __nv_bfloat16, true>(a, stream) : launch<false, __nv_bfloat16, true>(a, stream);
+  return kda ? launch<true, float, true>(a, stream) : launch<false, float, true>(a, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

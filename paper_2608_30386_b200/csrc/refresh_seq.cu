@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(DV *RS) refresh_seq_kernel(DascRefreshArgs a) 
   const int r = blockIdx.x / (a.H_v * a.n_layers_in_call);
   const int hk = h / (a.H_v / a.H_k);
   const int layer = a.layer_begin + lc;
-  const int64_t t_begin = a.cu_seqlens[r];
+  const int64_t t_begin = a.tok_begin ? a.tok_begin[r] : a.cu_seqlens[r];
   const int n_tok = static_cast<int>(a.cu_seqlens[r + 1] - t_begin);
   // An empty suffix continues nothing; in the scratch mode it still replaces the omitted
   // units by the (all-zero) scratch state, as the definition says.
