@@ -162,6 +162,30 @@ def restore(mask, unit_words, pool, slot_stride, src_slot, state, layer_stride, 
                          C.c_int32(src_slot.size))
 
 
+def pack_padded(mask, unit_words, state, layer_stride, req_stride, src_req, pool, n_slots, R_max, dst_slot):
+    """Appendix B padded layout: ``pool`` is [L][n_slots][R_max][unit_words]; padding is not written."""
+    mask = np.ascontiguousarray(mask, np.uint8)
+    L, n_l = mask.shape
+    src_req = np.ascontiguousarray(src_req, np.int32)
+    dst_slot = np.ascontiguousarray(dst_slot, np.int32)
+    assert pool.size >= L * n_slots * R_max * unit_words
+    lib().oracle_pack_padded(_p(mask), C.c_int32(L), C.c_int64(n_l), C.c_int64(unit_words), _p(_words(state)),
+                             C.c_int64(layer_stride), C.c_int64(req_stride), _p(src_req), _p(_words(pool)),
+                             C.c_int64(n_slots), C.c_int64(R_max), _p(dst_slot), C.c_int32(src_req.size))
+
+
+def restore_padded(mask, unit_words, pool, n_slots, R_max, src_slot, state, layer_stride, req_stride, dst_req):
+    """Zero-fill load from the padded pool (in place on ``state``)."""
+    mask = np.ascontiguousarray(mask, np.uint8)
+    L, n_l = mask.shape
+    src_slot = np.ascontiguousarray(src_slot, np.int32)
+    dst_req = np.ascontiguousarray(dst_req, np.int32)
+    lib().oracle_restore_padded(_p(mask), C.c_int32(L), C.c_int64(n_l), C.c_int64(unit_words), _p(_words(pool)),
+                                C.c_int64(n_slots), C.c_int64(R_max), _p(src_slot), _p(_words(state)),
+                                C.c_int64(layer_stride), C.c_int64(req_stride), _p(dst_req),
+                                C.c_int32(src_slot.size))
+
+
 def refresh(kind, n_layers, H_v, H_k, d_k, d_v, state, layer_stride, req_stride, req_idx,
             q, k, v, g, beta, cu_seqlens, *, q_scale=1.0, want_o=True, mode=MODE_CONTINUE,
             mask=None, want_state64=False, n_threads=0):

@@ -320,6 +320,55 @@ void oracle_restore(const uint8_t *mask, int32_t n_layers, int64_t n_l, int64_t 
 }
 
 /* ------------------------------------------------------------------ */
+/* Appendix B, padded layout (Scheme 1): pool [L][slots][R_max][unit]   */
+/* ------------------------------------------------------------------ */
+
+/* Entry (l, slot, j) of the padded pool, j < R_max, starts at word
+ *     ((l*n_slots + slot)*R_max + j)*unit_words.
+ * Layer l's j-th retained unit (ascending unit index) goes to entry j; entries
+ * r_l .. R_max-1 are padding and are neither written (pack) nor read (restore). */
+void oracle_pack_padded(const uint8_t *mask, int32_t n_layers, int64_t n_l, int64_t unit_words,
+                        const uint32_t *state, int64_t layer_stride, int64_t req_stride,
+                        const int32_t *src_req, uint32_t *pool, int64_t n_slots, int64_t R_max,
+                        const int32_t *dst_slot, int32_t n_pairs)
+{
+    for (int32_t i = 0; i < n_pairs; ++i) {
+        for (int32_t l = 0; l < n_layers; ++l) {
+            int64_t j = 0; /* rank of the unit among the layer's retained units */
+            for (int64_t u = 0; u < n_l; ++u) {
+                if (!mask[l * n_l + u]) continue;
+                const uint32_t *src = state + (int64_t)src_req[i] * req_stride + l * layer_stride + u * unit_words;
+                uint32_t *dst = pool + (((int64_t)l * n_slots + dst_slot[i]) * R_max + j) * unit_words;
+                for (int64_t w = 0; w < unit_words; ++w) dst[w] = src[w];
+                ++j;
+            }
+        }
+    }
+}
+
+/* Zero-fill load from the padded pool: clear, then copy the valid entries back. */
+void oracle_restore_padded(const uint8_t *mask, int32_t n_layers, int64_t n_l, int64_t unit_words,
+                           const uint32_t *pool, int64_t n_slots, int64_t R_max, const int32_t *src_slot,
+                           uint32_t *state, int64_t layer_stride, int64_t req_stride,
+                           const int32_t *dst_req, int32_t n_pairs)
+{
+    for (int32_t i = 0; i < n_pairs; ++i) {
+        for (int32_t l = 0; l < n_layers; ++l) {
+            uint32_t *dense = state + (int64_t)dst_req[i] * req_stride + l * layer_stride;
+            for (int64_t w = 0; w < n_l * unit_words; ++w) dense[w] = 0u;
+            int64_t j = 0;
+            for (int64_t u = 0; u < n_l; ++u) {
+                if (!mask[l * n_l + u]) continue;
+                const uint32_t *src = pool + (((int64_t)l * n_slots + src_slot[i]) * R_max + j) * unit_words;
+                uint32_t *dst = dense + u * unit_words;
+                for (int64_t w = 0; w < unit_words; ++w) dst[w] = src[w];
+                ++j;
+            }
+        }
+    }
+}
+
+/* ------------------------------------------------------------------ */
 /* Suffix refresh (Section 3.1 Eq. 1; Section 4.2): token-by-token replay */
 /* ------------------------------------------------------------------ */
 

@@ -293,6 +293,52 @@ def test_round_trip_all_retained_is_bit_exact():
     np.testing.assert_array_equal(out.view(np.uint32), state.view(np.uint32))
 
 
+@pytest.mark.parametrize("unit_words,n_l", [(8, 24), (32, 5)])
+def test_padded_layout_holds_the_ragged_values_at_padded_positions(unit_words, n_l):
+    # Appendix B: pool [L][slots][R_max][unit]; the first r_l entries of layer l are the layer's retained units in
+    # order (the same values the ragged layout stores at [o_l, o_{l+1})), the rest is padding nobody touches.
+    rng = np.random.default_rng(6)
+    L, n_req, n_slots = 4, 4, 5
+    mask = (rng.random((L, n_l)) < 0.4).astype(np.uint8)
+    mask[2] = 0
+    mask[3, : n_l // 2 + 1] = 1                      # a heavy layer sets R_max
+    r_l = mask.sum(1)
+    R_max, sum_r = int(r_l.max()), int(r_l.sum())
+    layer_stride = n_l * unit_words + 8
+    req_stride = L * layer_stride + 16
+    state = _state_with_specials(rng, (n_req * req_stride,))
+    src_req = np.array([3, 0, 1], np.int32)
+    slots = np.array([4, 0, 2], np.int32)
+    padded = np.full((L, n_slots, R_max, unit_words), np.float32(7.0))
+    oracle.pack_padded(mask, unit_words, state, layer_stride, req_stride, src_req, padded, n_slots, R_max, slots)
+    ragged = np.zeros((n_slots, sum_r * unit_words), np.float32)
+    oracle.pack(mask, unit_words, state, layer_stride, req_stride, src_req, ragged, sum_r * unit_words, slots)
+    o_l = np.concatenate([[0], np.cumsum(r_l)])
+    pb, rb = padded.view(np.uint32), ragged.view(np.uint32).reshape(n_slots, sum_r, unit_words)
+    for s in range(n_slots):
+        for l in range(L):
+            if s in slots:
+                np.testing.assert_array_equal(pb[l, s, : r_l[l]], rb[s, o_l[l]: o_l[l + 1]])
+                # and directly from the definition: the masked rows of the dense layer
+                req = src_req[list(slots).index(s)]
+                dense = state.view(np.uint32)[req * req_stride + l * layer_stride:][: n_l * unit_words]
+                np.testing.assert_array_equal(pb[l, s, : r_l[l]], dense.reshape(n_l, unit_words)[mask[l].astype(bool)])
+                assert np.all(padded[l, s, r_l[l]:] == np.float32(7.0))      # padding untouched
+            else:
+                assert np.all(padded[l, s] == np.float32(7.0))
+    # loading from either layout gives the same dense state, bit for bit
+    dst_req = np.array([1, 2, 0], np.int32)
+    a = np.full_like(state, np.float32(-3.0))
+    b = np.full_like(state, np.float32(-3.0))
+    oracle.restore_padded(mask, unit_words, padded, n_slots, R_max, slots, a, layer_stride, req_stride, dst_req)
+    oracle.restore(mask, unit_words, ragged, sum_r * unit_words, slots, b, layer_stride, req_stride, dst_req)
+    np.testing.assert_array_equal(a.view(np.uint32), b.view(np.uint32))
+    # Appendix B capacity identities: C_rag / C_pad = R_max / mean(r_l)
+    plan_like_rag = (L * n_l) / sum_r
+    plan_like_pad = (L * n_l) / (L * R_max)
+    assert plan_like_rag / plan_like_pad == pytest.approx(R_max / r_l.mean())
+
+
 # ----------------------------------------------------------------------------
 # Eq. 1: the recurrence
 # ----------------------------------------------------------------------------
