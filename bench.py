@@ -141,11 +141,12 @@ def oracle_leg(c, sample_req=4, sample_units=64):
     L, H_v, H_k = c["L"], c["H_v"], c["H_k"]
     uph = D if kda else 1
     gen = synth.generator(c["seed"])
-    rates = synth.decay_rates(gen, L, H_v, uph, c["rate_lo"], 1.0)
+    rates = synth.skew_layers(synth.decay_rates(gen, L, H_v, uph, c["rate_lo"], 1.0), c.get("layer_skew", 0.0))
     A_log, dt = synth.decay_params(rates)
     unit_words = D if kda else D * D
     oplan = oracle.plan(okind, L, H_v, uph, A_log.numpy(), dt.numpy(), sel=oracle.SEL_TOP_RATIO,
-                        keep_ratio=c["keep"], scope=oracle.SCOPE_LAYER, unit_bytes=unit_words * 4)
+                        keep_ratio=c["keep"], unit_bytes=unit_words * 4,
+                        scope=oracle.SCOPE_MODEL if c.get("scope") == "model" else oracle.SCOPE_LAYER)
     dense = H_v * D * D
     state = synth.states(gen, (sample_req, L, dense)).numpy()
     slot = oplan.sum_r * unit_words
@@ -220,10 +221,12 @@ def build_plan(c, device):
     from paper_2608_30386_b200 import synth
     kda = c["kind"] == "KDA"
     gen = synth.generator(c["seed"])
-    rates = synth.decay_rates(gen, c["L"], c["H_v"], D if kda else 1, c["rate_lo"], 1.0)
+    rates = synth.skew_layers(synth.decay_rates(gen, c["L"], c["H_v"], D if kda else 1, c["rate_lo"], 1.0),
+                              c.get("layer_skew", 0.0))
     A_log, dt = synth.decay_params(rates)
     plan = dasc.dasc_plan(dasc.KDA if kda else dasc.GDN, c["L"], c["H_v"], c["H_k"], D, D, A_log.numpy(), dt.numpy(),
-                          sel=dasc.SEL_TOP_RATIO, scope=dasc.SCOPE_LAYER, keep_ratio=c["keep"], device=device)
+                          sel=dasc.SEL_TOP_RATIO, scope=dasc.SCOPE_MODEL if c.get("scope") == "model" else dasc.SCOPE_LAYER,
+                          keep_ratio=c["keep"], device=device)
     return plan, rates, gen
 
 
@@ -247,6 +250,12 @@ def main():
     ap.add_argument("--suffix", type=int, default=None, help="refresh suffix length (config 3: 256, 1024, 4096)")
     ap.add_argument("--keep", type=float, default=None, help="keep ratio (0.25, 0.38, 0.5, 1.0 in the sweep)")
     ap.add_argument("--layer-group", type=int, default=None, help="layers of token streams resident at once")
+    ap.add_argument("--layout", default="ragged", choices=["ragged", "padded"],
+                    help="checkpoint pool layout (Appendix B): ragged [slots][sum r_l] or padded [L][slots][R_max]")
+    ap.add_argument("--scope", default="layer", choices=["layer", "model"],
+                    help="selection scope of the keep ratio; 'model' makes per-layer counts differ (padding appears)")
+    ap.add_argument("--layer-skew", type=float, default=0.0,
+                    help="imbalanced per-layer decay profile: layer rates scaled by exp(skew * (l/(L-1) - 1/2))")
     ap.add_argument("--codec", default="fp32", choices=["fp32", "int8"],
                     help="checkpoint pool format: fp32 bit copies, or the Appendix D INT8 codec fused into pack/restore")
     args = ap.parse_args()
@@ -258,6 +267,8 @@ def main():
     if args.keep is not None:
         c["keep"] = args.keep
     c["codec"] = args.codec
+    c["scope"] = args.scope
+    c["layer_skew"] = args.layer_skew
     if args.impl == "reference":
         run_reference(args, c)
         return
@@ -298,6 +309,16 @@ def main():
     pool = torch.empty((N_REQ, slot_bytes), dtype=torch.uint8, device=dev) if int8 else torch.empty((N_REQ, slot), device=dev)
     do_pack = dasc.dasc_pack_int8 if int8 else dasc.dasc_pack
     do_restore = dasc.dasc_restore_int8 if int8 else dasc.dasc_restore
+    if args.layout == "padded":                                # Appendix B, Scheme 1: [L][slots][R_max][unit]
+        if int8:
+            raise SystemExit("--layout padded is an fp32 layout")
+        pool = torch.empty(dasc.dasc_padded_pool_floats(plan, N_REQ), device=dev)
+
+        def do_pack(plan, state, ls, rs, src, pool, dst):
+            dasc.dasc_pack_padded(plan, state, ls, rs, src, pool, int(dst.numel()), dst)
+
+        def do_restore(plan, pool, src, state, ls, rs, dst):
+            dasc.dasc_restore_padded(plan, pool, int(src.numel()), src, state, ls, rs, dst)
     ids = torch.arange(N_REQ, dtype=torch.int32, device=dev)
     slots = torch.randperm(N_REQ, generator=gen).to(torch.int32).to(dev)
     T = N_REQ * SUFFIX
@@ -498,7 +519,8 @@ def main():
         "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_total,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(c), "kind": c["kind"], "layers": L, "v_heads": H_v, "k_heads": H_k, "d_k": D,
-                   "d_v": D, "requests": N_REQ, "keep_ratio": c["keep"], "codec": args.codec, "suffix_tokens": SUFFIX, "refresh_algo": args.algo,
+                   "d_v": D, "requests": N_REQ, "keep_ratio": c["keep"], "codec": args.codec, "layout": args.layout, "selection_scope": args.scope,
+                   "pool_bytes": pool.numel() * pool.element_size(), "suffix_tokens": SUFFIX, "refresh_algo": args.algo,
                    "stream_layers_resident": group,
                    "l2": "inputs larger than L2 (GiBs of states and token streams per step); no flush needed",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
@@ -506,6 +528,16 @@ def main():
         "pack_GBps": world * pack_gbs, "restore_GBps": world * restore_gbs,
         "refresh_tokens_per_s": world * N_REQ * SUFFIX / (t_refresh * 1e-3),
         "refresh_token_heads_per_s": world * token_heads / (t_refresh * 1e-3),
+        # Eq. 6 / Appendix B on this plan: temporal bytes of one checkpoint per layout and the layout gain R_max / mean r_l
+        "capacity": {
+            "layer_skew": args.layer_skew,
+            "bytes_dense": dasc.dasc_checkpoint_bytes(plan, dasc.LAYOUT_DENSE),
+            "bytes_padded": dasc.dasc_checkpoint_bytes(plan, dasc.LAYOUT_PADDED),
+            "bytes_ragged": dasc.dasc_checkpoint_bytes(plan, dasc.LAYOUT_RAGGED),
+            "bytes_ragged_int8": dasc.dasc_int8_slot_bytes(plan),
+            "c_temp_pad": plan.c_temp_pad, "c_temp_rag": plan.c_temp_rag,
+            "layout_gain_rmax_over_rbar": plan.c_temp_rag / plan.c_temp_pad if plan.units_retained else None,
+        },
         # dasc_refresh_window: scratch replay of the last `suffix_tokens` tokens, merge of omitted units, no outputs
         "window_refresh_state_only": {"ms": t_window, "tokens_per_s": world * N_REQ * SUFFIX / (t_window * 1e-3),
                                       "token_heads_per_s": world * token_heads / (t_window * 1e-3)},

@@ -186,6 +186,45 @@ dasc_status_t dasc_restore(const dasc_plan_t *plan, const float *pool_base, int6
                            void *cuda_stream);
 
 /*
+ * Padded checkpoint layout (Appendix B, Scheme 1), the paper's comparison point for
+ * the ragged layout: one contiguous pool [n_layers][n_slots][R_max][unit_floats]
+ * fp32 with R_max = max_l r_l; entry (l, slot, j) holds the j-th retained unit of
+ * layer l (ascending unit index) for j < r_l, and entries r_l .. R_max-1 are
+ * padding that dasc_pack_padded never writes and dasc_restore_padded never reads.
+ * The retained values are those of the ragged layout, so loading from either
+ * layout gives the same state.
+ *   dasc_padded_pool_floats  floats of such a pool for n_slots slots.
+ *   pool_base  DEVICE, 16-byte aligned, at least that many floats.
+ *   n_slots    the pool's slot count (> 0); slot indices must be < n_slots.
+ * Everything else as for dasc_pack / dasc_restore.
+ */
+dasc_status_t dasc_padded_pool_floats(const dasc_plan_t *plan, int64_t n_slots, int64_t *out);
+dasc_status_t dasc_pack_padded(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride,
+                               int64_t req_stride, const int32_t *src_req, float *pool_base,
+                               int64_t n_slots, const int32_t *dst_slot, int32_t n_pairs,
+                               void *cuda_stream);
+dasc_status_t dasc_restore_padded(const dasc_plan_t *plan, const float *pool_base, int64_t n_slots,
+                                  const int32_t *src_slot, float *state_base, int64_t layer_stride,
+                                  int64_t req_stride, const int32_t *dst_req, int32_t n_pairs,
+                                  void *cuda_stream);
+
+/*
+ * Complete-checkpoint accounting (host arithmetic only).
+ * dasc_checkpoint_bytes: bytes of one checkpoint under a layout, temporal state
+ *   plus the uncompressed convolution state B_conv that is stored alongside
+ *   (Eq. 6, Appendix B): ragged sum_l r_l units, padded L * R_max units, dense
+ *   sum_l n_l units, each unit_floats * 4 bytes, + conv_bytes.  Ratios of these
+ *   are C_ckpt; dense / padded and dense / ragged differ by R_max / mean(r_l).
+ * dasc_slot_budget (Appendix C.1): with per-rank temporal bytes b_r and the
+ *   convolution bytes b_conv, N = floor(B / max_r (b_r + b_conv)) - 1; one slot
+ *   is reserved by the allocator.  HOST pointers.
+ */
+typedef enum { DASC_LAYOUT_RAGGED = 0, DASC_LAYOUT_PADDED = 1, DASC_LAYOUT_DENSE = 2 } dasc_layout_t;
+dasc_status_t dasc_checkpoint_bytes(const dasc_plan_t *plan, int32_t layout, int64_t conv_bytes, int64_t *out);
+dasc_status_t dasc_slot_budget(int64_t budget_bytes, const int64_t *temporal_bytes_per_rank,
+                               int32_t n_ranks, int64_t conv_bytes, int64_t *out);
+
+/*
  * INT8 checkpoint codec fused into the Store / Load copies (Appendix D, Eq. 10).
  * A row is the d_v values of one (layer, head, key channel) tuple; rows are the
  * plan's retained rows in ragged order (a retained GDN head contributes its d_k

@@ -30,6 +30,7 @@ EXPORTS = (
     "dasc_plan", "dasc_plan_destroy", "dasc_plan_info", "dasc_plan_horizon", "dasc_plan_mask",
     "dasc_plan_window", "dasc_plan_layer_counts", "dasc_plan_layer_offsets", "dasc_pack", "dasc_restore",
     "dasc_int8_slot_bytes", "dasc_pack_int8", "dasc_restore_int8",
+    "dasc_padded_pool_floats", "dasc_pack_padded", "dasc_restore_padded", "dasc_checkpoint_bytes", "dasc_slot_budget",
     "dasc_refresh_workspace_bytes", "dasc_refresh", "dasc_refresh_status", "dasc_refresh_window", "dasc_refresh_static",
     "dasc_status_string", "dasc_version",
 )
@@ -90,6 +91,11 @@ def lib() -> C.CDLL:
                                 C.c_void_p, C.c_int32, C.c_void_p]
         L.dasc_restore.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                    C.c_void_p, C.c_int32, C.c_void_p]
+        L.dasc_padded_pool_floats.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int64)]
+        L.dasc_pack_padded.argtypes = L.dasc_pack.argtypes
+        L.dasc_restore_padded.argtypes = L.dasc_restore.argtypes
+        L.dasc_checkpoint_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_int64)]
+        L.dasc_slot_budget.argtypes = [C.c_int64, C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_int64)]
         L.dasc_int8_slot_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
         L.dasc_pack_int8.argtypes = L.dasc_pack.argtypes
         L.dasc_restore_int8.argtypes = L.dasc_restore.argtypes
@@ -224,6 +230,48 @@ def dasc_restore(plan: Plan, pool: torch.Tensor, src_slot: torch.Tensor, state: 
     """Scatter pool slots ``src_slot`` into the dense states ``dst_req``; omitted units become +0.0."""
     _check(lib().dasc_restore(plan.handle, _ptr(pool), slot_stride, _ptr(src_slot), _ptr(state), layer_stride,
                               req_stride, _ptr(dst_req), int(src_slot.numel()), _stream_ptr(stream)), "dasc_restore")
+
+
+LAYOUT_RAGGED, LAYOUT_PADDED, LAYOUT_DENSE = 0, 1, 2
+
+
+def dasc_padded_pool_floats(plan: Plan, n_slots: int) -> int:
+    """Floats of a padded pool [L][n_slots][R_max][unit_floats] (Appendix B, Scheme 1)."""
+    out = C.c_int64()
+    _check(lib().dasc_padded_pool_floats(plan.handle, int(n_slots), C.byref(out)), "dasc_padded_pool_floats")
+    return int(out.value)
+
+
+def dasc_pack_padded(plan: Plan, state: torch.Tensor, layer_stride: int, req_stride: int, src_req: torch.Tensor,
+                     pool: torch.Tensor, n_slots: int, dst_slot: torch.Tensor, stream=None):
+    """``dasc_pack`` into the padded pool; padding entries are not written."""
+    _check(lib().dasc_pack_padded(plan.handle, _ptr(state), layer_stride, req_stride, _ptr(src_req), _ptr(pool),
+                                  int(n_slots), _ptr(dst_slot), int(src_req.numel()), _stream_ptr(stream)),
+           "dasc_pack_padded")
+
+
+def dasc_restore_padded(plan: Plan, pool: torch.Tensor, n_slots: int, src_slot: torch.Tensor, state: torch.Tensor,
+                        layer_stride: int, req_stride: int, dst_req: torch.Tensor, stream=None):
+    """``dasc_restore`` from the padded pool."""
+    _check(lib().dasc_restore_padded(plan.handle, _ptr(pool), int(n_slots), _ptr(src_slot), _ptr(state), layer_stride,
+                                     req_stride, _ptr(dst_req), int(src_slot.numel()), _stream_ptr(stream)),
+           "dasc_restore_padded")
+
+
+def dasc_checkpoint_bytes(plan: Plan, layout: int, conv_bytes: int = 0) -> int:
+    """Bytes of one checkpoint (temporal state under ``layout`` + convolution state), Eq. 6 / Appendix B."""
+    out = C.c_int64()
+    _check(lib().dasc_checkpoint_bytes(plan.handle, int(layout), int(conv_bytes), C.byref(out)), "dasc_checkpoint_bytes")
+    return int(out.value)
+
+
+def dasc_slot_budget(budget_bytes: int, temporal_bytes_per_rank, conv_bytes: int = 0) -> int:
+    """Appendix C.1: N = floor(B / max_r(b_r + b_conv)) - 1."""
+    arr = np.ascontiguousarray(temporal_bytes_per_rank, np.int64)
+    out = C.c_int64()
+    _check(lib().dasc_slot_budget(int(budget_bytes), arr.ctypes.data_as(C.c_void_p), int(arr.size), int(conv_bytes),
+                                  C.byref(out)), "dasc_slot_budget")
+    return int(out.value)
 
 
 def dasc_int8_slot_bytes(plan: Plan) -> int:

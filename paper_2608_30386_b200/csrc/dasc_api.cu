@@ -39,6 +39,8 @@ void free_device_tables(dasc_plan_s *p) {
   cudaFree(p->d_row_src);
   cudaFree(p->d_row_pos);
   cudaFree(p->d_row_keep);
+  cudaFree(p->d_layer_row_off);
+  p->d_layer_row_off = nullptr;
   p->d_row_src = nullptr;
   p->d_row_pos = nullptr;
   p->d_row_keep = nullptr;
@@ -111,6 +113,11 @@ dasc_status_t dasc_plan(const dasc_plan_desc_t *desc, int32_t device, dasc_plan_
     cudaError_t e = upload(&p->d_row_src, p->row_src.data(), p->row_src.size());
     if (e == cudaSuccess) e = upload(&p->d_row_pos, p->row_pos.data(), p->row_pos.size());
     if (e == cudaSuccess) e = upload(&p->d_row_keep, keep.data(), keep.size());
+    // packed row at which each layer starts: o_l in rows (a GDN unit is d_k rows)
+    const int64_t rows_per_unit = p->info.unit_floats / p->info.d_v;
+    std::vector<int32_t> row_off(p->layer_offset.size());
+    for (size_t l = 0; l < row_off.size(); ++l) row_off[l] = static_cast<int32_t>(p->layer_offset[l] * rows_per_unit);
+    if (e == cudaSuccess) e = upload(&p->d_layer_row_off, row_off.data(), row_off.size());
     if (e != cudaSuccess) {
       free_device_tables(p);
       delete p;
@@ -165,6 +172,66 @@ dasc_status_t dasc_restore(const dasc_plan_t *plan, const float *pool_base, int6
   const int e = dasc_launch_restore(plan, pool_base, slot_stride, src_slot, state_base, layer_stride, req_stride,
                                     dst_req, n_pairs, cuda_stream);
   return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+dasc_status_t dasc_padded_pool_floats(const dasc_plan_t *plan, int64_t n_slots, int64_t *out) {
+  if (!plan || !out || n_slots < 0) return DASC_ERR_INVALID_ARG;
+  *out = static_cast<int64_t>(plan->info.n_layers) * n_slots * plan->info.r_max * plan->info.unit_floats;
+  return DASC_OK;
+}
+
+dasc_status_t dasc_pack_padded(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride,
+                               int64_t req_stride, const int32_t *src_req, float *pool_base, int64_t n_slots,
+                               const int32_t *dst_slot, int32_t n_pairs, void *cuda_stream) {
+  int64_t unused = 0;
+  dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, src_req, pool_base, &unused, dst_slot,
+                                     n_pairs);
+  if (st != DASC_OK || n_pairs == 0) return st;
+  if (n_slots <= 0) return DASC_ERR_INVALID_ARG;
+  const int e = dasc_launch_pack_padded(plan, state_base, layer_stride, req_stride, src_req, pool_base, n_slots,
+                                        dst_slot, n_pairs, cuda_stream);
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+dasc_status_t dasc_restore_padded(const dasc_plan_t *plan, const float *pool_base, int64_t n_slots,
+                                  const int32_t *src_slot, float *state_base, int64_t layer_stride,
+                                  int64_t req_stride, const int32_t *dst_req, int32_t n_pairs, void *cuda_stream) {
+  int64_t unused = 0;
+  dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, dst_req, pool_base, &unused, src_slot,
+                                     n_pairs);
+  if (st != DASC_OK || n_pairs == 0) return st;
+  if (n_slots <= 0) return DASC_ERR_INVALID_ARG;
+  const int e = dasc_launch_restore_padded(plan, pool_base, n_slots, src_slot, state_base, layer_stride, req_stride,
+                                           dst_req, n_pairs, cuda_stream);
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+dasc_status_t dasc_checkpoint_bytes(const dasc_plan_t *plan, int32_t layout, int64_t conv_bytes, int64_t *out) {
+  if (!plan || !out || conv_bytes < 0) return DASC_ERR_INVALID_ARG;
+  int64_t units;
+  switch (layout) {
+    case DASC_LAYOUT_RAGGED: units = plan->info.units_retained; break;
+    case DASC_LAYOUT_PADDED: units = static_cast<int64_t>(plan->info.n_layers) * plan->info.r_max; break;
+    case DASC_LAYOUT_DENSE: units = plan->info.units_total; break;
+    default: return DASC_ERR_INVALID_ARG;
+  }
+  *out = units * plan->info.unit_floats * 4 + conv_bytes;
+  return DASC_OK;
+}
+
+dasc_status_t dasc_slot_budget(int64_t budget_bytes, const int64_t *temporal_bytes_per_rank, int32_t n_ranks,
+                               int64_t conv_bytes, int64_t *out) {
+  if (!temporal_bytes_per_rank || !out || n_ranks <= 0 || budget_bytes < 0 || conv_bytes < 0)
+    return DASC_ERR_INVALID_ARG;
+  int64_t bottleneck = 0;
+  for (int32_t r = 0; r < n_ranks; ++r) {
+    if (temporal_bytes_per_rank[r] < 0) return DASC_ERR_INVALID_ARG;
+    const int64_t b = temporal_bytes_per_rank[r] + conv_bytes;
+    if (b > bottleneck) bottleneck = b;
+  }
+  if (bottleneck == 0) return DASC_ERR_INVALID_ARG;
+  *out = budget_bytes / bottleneck - 1;  // slot 0 is reserved by the allocator
+  return DASC_OK;
 }
 
 static int64_t int8_slot_bytes(const dasc_plan_t *plan) {

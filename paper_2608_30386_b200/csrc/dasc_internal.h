@@ -29,6 +29,7 @@ struct dasc_plan_s {
   DascRowSrc *d_row_src = nullptr;
   int32_t *d_row_pos = nullptr;
   uint8_t *d_row_keep = nullptr;     // [L][rows_per_layer]: 1 = retained row
+  int32_t *d_layer_row_off = nullptr;  // [L+1]: packed row at which each layer starts
 };
 
 // plan_host.cpp
@@ -41,6 +42,14 @@ int dasc_launch_pack(const dasc_plan_s *plan, const float *state, int64_t layer_
 int dasc_launch_restore(const dasc_plan_s *plan, const float *pool, int64_t slot_stride, const int32_t *src_slot,
                         float *state, int64_t layer_stride, int64_t req_stride, const int32_t *dst_req,
                         int32_t n_pairs, void *stream);
+
+// pack_restore_padded.cu: pool [L][n_slots][R_max][unit]
+int dasc_launch_pack_padded(const dasc_plan_s *plan, const float *state, int64_t layer_stride, int64_t req_stride,
+                            const int32_t *src_req, float *pool, int64_t n_slots, const int32_t *dst_slot,
+                            int32_t n_pairs, void *stream);
+int dasc_launch_restore_padded(const dasc_plan_s *plan, const float *pool, int64_t n_slots, const int32_t *src_slot,
+                               float *state, int64_t layer_stride, int64_t req_stride, const int32_t *dst_req,
+                               int32_t n_pairs, void *stream);
 
 // codec_int8.cu
 int dasc_launch_pack_int8(const dasc_plan_s *plan, const float *state, int64_t layer_stride, int64_t req_stride,

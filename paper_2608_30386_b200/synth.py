@@ -35,6 +35,16 @@ def decay_rates(gen, n_layers, n_heads, units_per_head, lo, hi, device="cpu") ->
     return torch.exp(u * (math.log(hi) - math.log(lo)) + math.log(lo))
 
 
+def skew_layers(rates: torch.Tensor, skew: float) -> torch.Tensor:
+    """Imbalanced per-layer decay profile: layer l's rates are multiplied by exp(skew * (l/(L-1) - 1/2)), so the
+    first layers decay slowly (long horizons) and the last ones fast.  skew = 0 leaves the rates as drawn."""
+    L = rates.shape[0]
+    if skew == 0.0 or L < 2:
+        return rates
+    pos = torch.arange(L, dtype=torch.float32, device=rates.device) / (L - 1) - 0.5
+    return rates * torch.exp(skew * pos).view(L, *([1] * (rates.dim() - 1)))
+
+
 def decay_params(rates: torch.Tensor):
     """(A_log, dt_bias) such that exp(A_log) = rate and dt_bias = 0."""
     return torch.log(rates).to(torch.float32), torch.zeros_like(rates)

@@ -313,7 +313,7 @@ def test_padded_layout_holds_the_ragged_values_at_padded_positions(unit_words, n
     oracle.pack_padded(mask, unit_words, state, layer_stride, req_stride, src_req, padded, n_slots, R_max, slots)
     ragged = np.zeros((n_slots, sum_r * unit_words), np.float32)
     oracle.pack(mask, unit_words, state, layer_stride, req_stride, src_req, ragged, sum_r * unit_words, slots)
-    o_l = np.concatenate([[0], np.cumsum(r_l)])
+    o_l = np.concatenate([[0], np.cumsum(r_l)]).astype(np.int64)
     pb, rb = padded.view(np.uint32), ragged.view(np.uint32).reshape(n_slots, sum_r, unit_words)
     for s in range(n_slots):
         for l in range(L):

@@ -124,3 +124,33 @@ def test_plan_argument_errors():
     p = dasc.dasc_plan(dasc.KDA, 1, 2, 2, 8, 8, A, A, device=-1)
     st = dasc.lib().dasc_pack(p.handle, None, 0, 0, None, None, 0, None, 1, None)
     assert st == binding.ERR_INVALID_ARG
+
+
+def test_checkpoint_accounting_and_slot_budget_match_oracle_and_paper():
+    """Host arithmetic of Eq. 6 / Appendix B / Appendix C.1 against the oracle's plan and the paper's byte budgets."""
+    rng = np.random.default_rng(11)
+    L, H, d = 6, 4, 32
+    A_log = np.log(_rates(rng, (L, H, d)))
+    dt = np.zeros_like(A_log)
+    conv = 4096
+    p = dasc.dasc_plan(dasc.KDA, L, H, H, d, 64, A_log, dt, w_max=64.0, conv_bytes_per_ckpt=conv, device=-1)
+    o = oracle.plan(oracle.KDA, L, H, d, A_log, dt, w_max=64.0, unit_bytes=64 * 4, conv_bytes=conv)
+    rag = dasc.dasc_checkpoint_bytes(p, dasc.LAYOUT_RAGGED, conv)
+    pad = dasc.dasc_checkpoint_bytes(p, dasc.LAYOUT_PADDED, conv)
+    dense = dasc.dasc_checkpoint_bytes(p, dasc.LAYOUT_DENSE, conv)
+    assert rag == o.sum_r * 256 + conv and pad == L * o.R_max * 256 + conv and dense == o.sum_n * 256 + conv
+    assert dense / rag == pytest.approx(o.C_ckpt_rag, rel=1e-14)
+    # temporal-only ratios: the layout gain is R_max / mean(r_l)
+    t = [dasc.dasc_checkpoint_bytes(p, lay, 0) for lay in (dasc.LAYOUT_RAGGED, dasc.LAYOUT_PADDED, dasc.LAYOUT_DENSE)]
+    assert t[2] / t[0] == pytest.approx(o.C_temp_rag) and t[2] / t[1] == pytest.approx(o.C_temp_pad)
+    assert t[1] / t[0] == pytest.approx(o.R_max / o.r_l.mean())
+    assert dasc.dasc_padded_pool_floats(p, 7) == L * 7 * o.R_max * 64
+    # slot budget: the oracle's function on the same inputs, and the paper's dense budgets (128 slots -> 127)
+    for budget, per_rank, cv in ((1000, [90, 240, 10], 10), (694681600, [5242880] * 8, 184320),
+                                 (1236271104, [9437184] * 8, 221184)):
+        assert dasc.dasc_slot_budget(budget, per_rank, cv) == oracle.slot_budget(budget, per_rank, cv)
+    assert dasc.dasc_slot_budget(694681600, [20 * 32 * 128 * 128 * 4 // 8] * 8, 20 * 3 * (3 * 32 * 128) // 8 * 2) == 127
+    with pytest.raises(dasc.DascError):
+        dasc.dasc_checkpoint_bytes(p, 9, 0)
+    with pytest.raises(dasc.DascError):
+        dasc.dasc_slot_budget(100, [0, 0], 0)
