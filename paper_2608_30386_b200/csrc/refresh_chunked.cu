@@ -1,5 +1,5 @@
-// Suffix refresh, chunked form, on the Blackwell tensor cores (tcgen05 + TMEM):
-// 32-token chunks, two CTAs resident per SM.
+// Suffix refresh, chunked form, on the Blackwell tensor cores (tcgen05 + TMEM), warp-specialised:
+// 32-token chunks, two CTAs resident per SM, three roles per CTA.
 //
 // Eq. 1 (transposed orientation) over a chunk of C = 32 tokens starting from S_0, with
 // G_t the running sum of the log-decay inside the chunk and m the chunk midpoint:
@@ -9,25 +9,19 @@
 //   U    = (I + A)^-1 * beta * (V - Kt S')                      (the deltas written at each token)
 //   O    = Qt S' + P U
 //   S_C  = Diag(exp(G_C - G_m)) (S' + Kh^T U)
-// Referencing the decay to the midpoint keeps every exponent within half a chunk's decay.
 //
-// Mapping.  One CTA per (request, layer, value head): eight compute warps (two per TMEM lane quadrant,
-// each taking half of the columns) and one warp that only issues tensor-core work; 256 TMEM columns and about 108 KB of shared memory per CTA, so two
-// CTAs share an SM and one fills the other's latency gaps (every phase of a chunk depends on the
-// one before it).  The state lives in TMEM transposed, S'^T: lane = value column v, column = key
-// channel c, fp32, for the whole suffix; the tensor core reads it as a tf32 operand directly.
-// All products are M = 128 tcgen05.mma (kind::tf32, fp32 accumulate) with the value index on the
-// TMEM lanes, so that each accumulator is the A operand of the next product:
+// Roles.  The operand tiles Kt, Qt, Kh depend on the token inputs only, not on the state, so they
+// are built one chunk ahead by four PRODUCER warps that read q, k and the log-decay straight from
+// global memory (their latency is off the critical path).  Eight CHAIN warps carry the
+// state-dependent sequence: state rescale -> triangular inverse -> right-hand side -> deltas ->
+// outputs.  One warp issues all tensor-core work.  The groups meet only at mbarriers.
 //   MMA1  [Kt;Qt] Kh^T            -> A (lanes 0-31) and P (lanes 32-63)         smem x smem
 //   MMA2  S'^T [Kt;Qt]^T          -> R^T | (Qt S')^T                            tmem x smem
 //   MMA3  RHS^T T^T               -> U^T      (RHS as a tf32 high/low pair)     tmem x smem
 //   MMA4  (Qt S')^T += U^T P^T    -> O^T                                         tmem x smem
 //   MMA5  S'^T      += U^T Kh     -> state    (U as a tf32 high/low pair)       tmem x smem
-// Operands built on the CUDA cores are rounded to tf32 (round-to-nearest).  T = (I + A)^-1 is
-// formed by one warp: 16x16 diagonal blocks by fp32 substitution, the off-diagonal block by
-// mma.sync (tf32) products.  Token inputs of chunk n+1 are fetched with cp.async while chunk n
-// computes.  Kh[t][c] (needed by MMA1 only) shares its storage with the T and P tiles; the raw
-// log-decay tile shares its storage with the V tile.
+// Buffers: the Kt/Qt and Kh tiles of chunk n+1 may be written once MMA2 of chunk n has completed
+// (MMA1 and MMA2 are their only readers); Kh^T, read last (MMA5), is double-buffered by chunk parity.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -38,35 +32,35 @@ namespace {
 
 using namespace tc5;
 
-constexpr int C = 32;        // chunk length
-constexpr int D = 128;       // d_k = d_v
-constexpr int NC = 256;      // compute threads
-constexpr int NT = NC + 32;  // + the MMA-issuing warp
-constexpr int LDX = 36;      // row pitch (floats) of the fp32 triangular work matrices
+constexpr int C = 32;          // chunk length
+constexpr int D = 128;         // d_k = d_v
+constexpr int NCH = 256;       // chain threads (warps 0-7)
+constexpr int NP = 128;        // producer threads (warps 8-11)
+constexpr int WARP_T = 12;     // the warp that inverts the triangular system
+constexpr int WARP_MMA = 13;   // the warp that issues tensor-core work
+constexpr int NT = NCH + NP + 64;
+constexpr int LDX = 36;        // row pitch (floats) of the fp32 triangular work matrices
 constexpr uint32_t TMEM_COLS = 256;
 
 // TMEM columns
 constexpr uint32_t COL_S = 0, COL_AP = 128, COL_RO = 160, COL_U = 224;  // RO: R^T 160-191 | (Qt S')^T 192-223
 
 // shared memory map (bytes)
-constexpr uint32_t OFF_KQ = 0;                         // [4][64 rows][128 B]  rows 0-31 Kt, 32-63 Qt; later the O tile
-constexpr uint32_t OFF_KHT = OFF_KQ + 4 * 64 * 128;    // [1][128 rows][128 B] Kh^T[c][t]
-constexpr uint32_t OFF_KH = OFF_KHT + 128 * 128;       // [4][32 rows][128 B]  Kh[t][c], until MMA1 is done; then:
-constexpr uint32_t OFF_TM = OFF_KH;                    // [1][32 rows][128 B]  T[t][i]
-constexpr uint32_t OFF_PM = OFF_TM + 32 * 128;         // [1][32 rows][128 B]  P[t][i]
-constexpr uint32_t OFF_RAWQ = OFF_KH + 4 * 32 * 128;   // [32][128] bf16 raw q of the next chunk
-constexpr uint32_t OFF_RAWK = OFF_RAWQ + C * D * 2;    // [32][128] bf16 raw k of the next chunk
-constexpr uint32_t OFF_G = OFF_RAWK + C * D * 2;       // [32][128] fp32 raw g (until prep), then
-constexpr uint32_t OFF_V = OFF_G;                      // [32][128] bf16 v (until the right-hand side is formed)
-constexpr uint32_t OFF_L = OFF_G + C * D * 4;          // [32][LDX] fp32
-constexpr uint32_t OFF_X = OFF_L + C * LDX * 4;        // [32][LDX] fp32
-constexpr uint32_t OFF_FAC = OFF_X + C * LDX * 4;      // [128] fp32 state factor per channel
-constexpr uint32_t OFF_POST = OFF_FAC + D * 4;         // [2][128] fp32 log-factor owed after a chunk, by chunk parity
-constexpr uint32_t OFF_BETA = OFF_POST + 2 * D * 4;    // [2][32] fp32, by chunk parity
-constexpr uint32_t OFF_GSC = OFF_BETA + 2 * C * 4;     // [2][32] fp32 scalar log-decay (GDN), by chunk parity
-constexpr uint32_t OFF_MISC = OFF_GSC + 2 * C * 4;     // barriers, tmem base, abort flag
+constexpr uint32_t OFF_KQ = 0;                          // [4][64 rows][128 B]  rows 0-31 Kt, 32-63 Qt
+constexpr uint32_t OFF_KHT = OFF_KQ + 4 * 64 * 128;     // [2][128 rows][128 B] Kh^T[c][t], by chunk parity
+constexpr uint32_t OFF_KH = OFF_KHT + 2 * 128 * 128;    // [4][32 rows][128 B]  Kh[t][c]
+constexpr uint32_t OFF_TM = OFF_KH + 4 * 32 * 128;      // [1][32 rows][128 B]  T[t][i]; TM|PM later the bf16 O tile
+constexpr uint32_t OFF_PM = OFF_TM + 32 * 128;          // [1][32 rows][128 B]  P[t][i]
+constexpr uint32_t OFF_V = OFF_PM + 32 * 128;           // [32][128] bf16 v
+constexpr uint32_t OFF_L = OFF_V + C * D * 2;           // [32][LDX] fp32
+constexpr uint32_t OFF_X = OFF_L + C * LDX * 4;         // [32][LDX] fp32
+constexpr uint32_t OFF_FAC = OFF_X + C * LDX * 4;       // [2][128] fp32 state factor per channel, by chunk parity
+constexpr uint32_t OFF_POST = OFF_FAC + 2 * D * 4;      // [2][128] fp32 log-factor owed after a chunk, by chunk parity
+constexpr uint32_t OFF_BETA = OFF_POST + 2 * D * 4;     // [4][32] fp32, by chunk index mod 4 (written well ahead)
+constexpr uint32_t OFF_GSC = OFF_BETA + 4 * C * 4;      // [4][32] fp32 scalar log-decay (GDN), same ring
+constexpr uint32_t OFF_MISC = OFF_GSC + 4 * C * 4;      // barriers, tmem base, abort flag
 constexpr uint32_t SMEM_BYTES = OFF_MISC + 128;
-constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;     // slack to align the base to 1024 bytes
+constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;      // slack to align the base to 1024 bytes
 static_assert(SMEM_ALLOC <= 113 * 1024, "two CTAs per SM");
 
 constexpr uint32_t kMaxPolls = 1u << 22;
@@ -83,18 +77,28 @@ constexpr float kLog2TruncComp = 5.0774e-4f;  // log2(kTruncComp)
 #ifdef DASC_PHASE_TIMING
 #define PT_DECL long long pt_acc[16] = {0}; long long pt_last = clock64();
 #define PT(i) do { long long pt_now = clock64(); pt_acc[i] += pt_now - pt_last; pt_last = pt_now; } while (0)
-#define PT_DUMP do { if (blockIdx.x == gridDim.x / 2 && tid == 0) { long long *d = reinterpret_cast<long long *>(static_cast<char *>(a.workspace) + 64); for (int i = 0; i < 16; ++i) d[i] = pt_acc[i]; } } while (0)
+#define PT_DUMP(who, off) do { if (blockIdx.x == gridDim.x / 2 && (who)) { long long *d = reinterpret_cast<long long *>(static_cast<char *>(a.workspace) + 64) + (off); for (int i = 0; i < 16; ++i) d[i] = pt_acc[i]; } } while (0)
 #else
 #define PT_DECL
 #define PT(i)
-#define PT_DUMP
+#define PT_DUMP(who, off)
 #endif
 
 struct Misc {
-  // tensor core -> compute warps (one tcgen05.commit each per chunk)
+  // tensor core -> chain warps (one tcgen05.commit each per chunk); bar_ro also releases the producer
   uint64_t bar_ap, bar_ro, bar_u, bar_o, bar_s;
-  // compute warps -> issuing warp (256 arrivals each per chunk)
-  uint64_t rdy_prep, rdy_state, rdy_rhs, rdy_u;
+  // producer -> issuing warp and chain warps (128 arrivals per chunk)
+  uint64_t rdy_prep;
+  // producer -> chain warps: the state factors of a chunk are ready (128 arrivals per chunk)
+  // One barrier per chunk parity: the producer may hand over the factors of chunk n+1 before the chain warps
+  // have waited for those of chunk n, and a single barrier cannot tell phases two apart.
+  uint64_t rdy_fac[2];
+  // chain warps -> issuing warp (256 arrivals each per chunk)
+  uint64_t rdy_state, rdy_rhs, rdy_u;
+  // triangular warp -> chain warps (A has left TMEM: 32 arrivals) and -> issuing warp (T tile ready: 32 arrivals)
+  uint64_t a_taken, rdy_t;
+  // chain warps -> triangular warp: the T|P tile region is free again (256 arrivals per chunk)
+  uint64_t tp_free;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -110,12 +114,30 @@ __device__ __forceinline__ void cp_async16_zfill(uint32_t smem, const void *gmem
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem), "l"(gmem), "r"(n) : "memory");
 }
 
+__device__ __forceinline__ void cp_async8_zfill(uint32_t smem, const void *gmem, bool valid) {
+  const uint32_t n = valid ? 8u : 0u;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(smem), "l"(gmem), "r"(n) : "memory");
+}
+
+// non-blocking: has the phase of this parity completed?
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// barrier among the 256 compute threads only
-__device__ __forceinline__ void sync_compute() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// barrier among the 256 chain threads only
+__device__ __forceinline__ void sync_chain() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // Bounded wait; after one time-out every later wait of this CTA returns at once.
 __device__ __forceinline__ void wait_bar(uint64_t *bar, uint32_t parity, Misc *misc, uint32_t *err) {
@@ -163,6 +185,31 @@ __device__ __forceinline__ void warp_mm_store(float *Cb, const float (&acc)[2][4
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
+// packed pairs of fp32 (one instruction per pair)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+
 // WITH_O = false is the state-only variant (no outputs wanted): q is never read, the Qt rows, P and the
 // output product are left out.
 template <bool KDA, typename OT, bool WITH_O>
@@ -209,14 +256,19 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     mbar_init(&misc->bar_u, 1);
     mbar_init(&misc->bar_o, 1);
     mbar_init(&misc->bar_s, 1);
-    mbar_init(&misc->rdy_prep, NC);
-    mbar_init(&misc->rdy_state, NC);
-    mbar_init(&misc->rdy_rhs, NC);
-    mbar_init(&misc->rdy_u, NC);
+    mbar_init(&misc->rdy_prep, NP);
+    mbar_init(&misc->rdy_fac[0], NP);
+    mbar_init(&misc->rdy_fac[1], NP);
+    mbar_init(&misc->rdy_state, NCH);
+    mbar_init(&misc->rdy_rhs, NCH);
+    mbar_init(&misc->rdy_u, NCH);
+    mbar_init(&misc->a_taken, 32);
+    mbar_init(&misc->rdy_t, 32);
+    mbar_init(&misc->tp_free, NCH);
     misc->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 8) {
+  if (warp == WARP_MMA) {
     tmem_alloc(&misc->tmem_base, TMEM_COLS);
     tmem_relinquish();
   }
@@ -225,27 +277,32 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   tc_fence_after_sync();
   const uint32_t tm = misc->tmem_base;
   const int n_chunks = (n_tok + C - 1) / C;
+  constexpr float LOG2E = 1.4426950408889634f;
 
   constexpr uint32_t ID_N32 = idesc_tf32(128, 32, false, false);
   constexpr uint32_t ID_N64 = idesc_tf32(128, 64, false, false);
   constexpr uint32_t ID_N128 = idesc_tf32(128, 128, false, false);
 
-  if (warp == 8) {
+  if (warp == WARP_MMA) {
     // =========================== tensor-core issue warp ===========================
+    // MMA1: [Kt;Qt] Kh^T.  M is padded to 128: rows 64-127 of the A tile are whatever follows it in
+    // shared memory, and land in TMEM lanes 64-127 that nobody reads.
+    auto issue_mma1 = [&]() {
+      tc_fence_after_sync();
+#pragma unroll 1
+      for (int kk = 0; kk < 16; ++kk)  // K = 128 in slices of 8: block kk / 4, 32 bytes per slice inside a block
+        mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
+               desc_kmajor(sbase + OFF_KH + (kk >> 2) * (32 * 128) + (kk & 3) * 32), ID_N32, kk != 0);
+      mma_commit(&misc->bar_ap);
+    };
+    bool ahead = false;  // lane 0: MMA1 of this chunk went out during the previous one
     for (int ch = 0; ch < n_chunks; ++ch) {
       const uint32_t par = ch & 1;
-      // MMA1: [Kt;Qt] Kh^T.  M is padded to 128: rows 64-127 of the A tile are whatever follows it in
-      // shared memory, and land in TMEM lanes 64-127 that nobody reads.
-      if (lane == 0) wait_bar(&misc->rdy_prep, par, misc, err);
-      __syncwarp();
-      if (lane == 0) {
-        tc_fence_after_sync();
-#pragma unroll 1
-        for (int kk = 0; kk < 16; ++kk)  // K = 128 in slices of 8: block kk / 4, 32 bytes per slice inside a block
-          mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
-                 desc_kmajor(sbase + OFF_KH + (kk >> 2) * (32 * 128) + (kk & 3) * 32), ID_N32, kk != 0);
-        mma_commit(&misc->bar_ap);
+      if (lane == 0 && !ahead) {
+        wait_bar(&misc->rdy_prep, par, misc, err);
+        issue_mma1();
       }
+      __syncwarp();
       // MMA2: S'^T [Kt;Qt]^T, the fp32 state read as a tf32 operand
       if (lane == 0) wait_bar(&misc->rdy_state, par, misc, err);
       __syncwarp();
@@ -254,11 +311,14 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 #pragma unroll 1
         for (int kk = 0; kk < 16; ++kk)
           mma_ts(tm + COL_RO, tm + COL_S + kk * 8, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
-                 go ? ID_N64 : ID_N32, kk != 0);  // without outputs only the Kt rows are needed
+                 WITH_O ? ID_N64 : ID_N32, kk != 0);  // without outputs only the Kt rows are needed
         mma_commit(&misc->bar_ro);
       }
       // MMA3: U^T = RHS^T T^T; RHS^T is a tf32 pair (high part over R^T, low part in the A|P columns)
-      if (lane == 0) wait_bar(&misc->rdy_rhs, par, misc, err);
+      if (lane == 0) {
+        wait_bar(&misc->rdy_t, par, misc, err);
+        wait_bar(&misc->rdy_rhs, par, misc, err);
+      }
       __syncwarp();
       if (lane == 0) {
         tc_fence_after_sync();
@@ -267,13 +327,17 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           mma_ts(tm + COL_U, tm + (kk < 4 ? COL_RO : COL_AP) + (kk & 3) * 8, desc_kmajor(sbase + OFF_TM + (kk & 3) * 32),
                  ID_N32, kk != 0);
         mma_commit(&misc->bar_u);
+        // The A|P columns are free again (MMA3 was their last reader, and the tensor pipe runs in order): if the
+        // next chunk's tiles are ready, its MMA1 goes out now instead of behind this chunk's state update.
+        ahead = ch + 1 < n_chunks && !misc->abort_flag && mbar_test_wait(&misc->rdy_prep, par ^ 1);
+        if (ahead) issue_mma1();
       }
       // MMA4: O^T += U^T P^T (high part of U);  MMA5: S'^T += U^T Kh (U as a pair: high in place, low over RHS^T)
       if (lane == 0) wait_bar(&misc->rdy_u, par, misc, err);
       __syncwarp();
       if (lane == 0) {
         tc_fence_after_sync();
-        if (go) {
+        if (WITH_O) {
 #pragma unroll 1
           for (int kk = 0; kk < 4; ++kk)
             mma_ts(tm + COL_RO + 32, tm + COL_U + kk * 8, desc_kmajor(sbase + OFF_PM + kk * 32), ID_N32, true);
@@ -281,73 +345,279 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         mma_commit(&misc->bar_o);
 #pragma unroll 1
         for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tm + COL_S, tm + (kk < 4 ? COL_U : COL_RO) + (kk & 3) * 8, desc_kmajor(sbase + OFF_KHT + (kk & 3) * 32),
-                 ID_N128, true);
+          mma_ts(tm + COL_S, tm + (kk < 4 ? COL_U : COL_RO) + (kk & 3) * 8,
+                 desc_kmajor(sbase + OFF_KHT + par * (128 * 128) + (kk & 3) * 32), ID_N128, true);
         mma_commit(&misc->bar_s);
       }
       __syncwarp();
     }
+  } else if (warp == WARP_T) {
+    // ================================ triangular warp ================================
+    // T = (I + A)^-1 depends on the token inputs only, so it is formed off the chain: A out of TMEM (lanes 0-31 are
+    // this warp's quadrant), 16x16 diagonal blocks by fp32 substitution, the off-diagonal block by mma.sync products.
+    const uint32_t tlane = tm;  // TMEM lanes 0-31
+    for (int ch = 0; ch < n_chunks; ++ch) {
+      const uint32_t par = ch & 1;
+      const float *beta_c = beta_s + (ch & 3) * C;
+      wait_bar(&misc->bar_ap, par, misc, err);
+      tc_fence_after_sync();
+      uint32_t x[32];
+      tmem_ld32(tlane + COL_AP, x);
+      tmem_ld_wait();
+      tc_fence_before_sync();
+      mbar_arrive(&misc->a_taken);  // the chain warps may reuse the A|P columns
+      const int t = lane;
+      // row t of A = strict_lower(Kt Kh^T) * beta_t, kept in fp32 for the inverse
+      const float bt = beta_c[t] * kInvTruncComp;
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        float4 o;
+        o.x = (j + 0 < t) ? bt * __uint_as_float(x[j + 0]) : 0.f;
+        o.y = (j + 1 < t) ? bt * __uint_as_float(x[j + 1]) : 0.f;
+        o.z = (j + 2 < t) ? bt * __uint_as_float(x[j + 2]) : 0.f;
+        o.w = (j + 3 < t) ? bt * __uint_as_float(x[j + 3]) : 0.f;
+        *reinterpret_cast<float4 *>(Lm + t * LDX + j) = o;
+      }
+      __syncwarp();
+      // diagonal 16x16 blocks: lane (block b, column cc) solves (I + L_bb) x = e_cc by forward substitution
+      {
+        const int b = lane >> 4, cc = lane & 15;
+        const float *Lb = Lm + (b * 16) * LDX + b * 16;
+        float xs[16];
+#pragma unroll
+        for (int rr = 0; rr < 16; ++rr) {
+          float acc0 = (rr == cc) ? 1.f : 0.f, acc1 = 0.f;
+#pragma unroll
+          for (int j = 0; j + 1 < rr; j += 2) {
+            acc0 = fmaf(-Lb[rr * LDX + j], xs[j], acc0);
+            acc1 = fmaf(-Lb[rr * LDX + j + 1], xs[j + 1], acc1);
+          }
+          if (rr & 1) acc0 = fmaf(-Lb[rr * LDX + rr - 1], xs[rr - 1], acc0);
+          xs[rr] = acc0 + acc1;
+        }
+#pragma unroll
+        for (int rr = 0; rr < 16; ++rr) Xm[(b * 16 + rr) * LDX + b * 16 + cc] = xs[rr];
+      }
+      __syncwarp();
+      // off-diagonal block: X_10 = -X_11 (L_10 X_00); the product L_10 X_00 is parked in the unused block (0,1)
+      {
+        float acc[2][4] = {};
+        warp_mm_acc(acc, Lm + 16 * LDX, Xm, lane);
+        warp_mm_store(Xm + 16, acc, 1.f, lane);
+        __syncwarp();
+        float acc2[2][4] = {};
+        warp_mm_acc(acc2, Xm + 16 * LDX + 16, Xm + 16, lane);
+        warp_mm_store(Xm + 16 * LDX, acc2, -1.f, lane);
+      }
+      __syncwarp();
+      // the T tile's storage (shared with the P tile and the chain warps' output tile) is free once the chain
+      // warps have copied the previous chunk's outputs out
+      if (ch > 0) wait_bar(&misc->tp_free, par ^ 1, misc, err);
+      // T (lower triangle of X, unit diagonal) -> tf32 operand tile; lane = row
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        const float4 xv = *reinterpret_cast<const float4 *>(Xm + t * LDX + j);
+        uint4 o;
+        o.x = (j + 0 <= t) ? tf32_pre(xv.x) : 0u;
+        o.y = (j + 1 <= t) ? tf32_pre(xv.y) : 0u;
+        o.z = (j + 2 <= t) ? tf32_pre(xv.z) : 0u;
+        o.w = (j + 3 <= t) ? tf32_pre(xv.w) : 0u;
+        *reinterpret_cast<uint4 *>(smem + OFF_TM + sw128_offset(32, t, j)) = o;
+      }
+      fence_smem_to_async();
+      mbar_arrive(&misc->rdy_t);  // -> MMA3
+      __syncwarp();
+    }
+  } else if (warp >= 8) {
+    // =============================== producer warps ===============================
+    // warp = block of 32 channels; per half of the chunk, lane = (4 adjacent channels, 4 consecutive tokens), a 4 x 4
+    // tile, so that Kh can also be stored transposed.  The midpoint is the end of the first half: first-half
+    // exponents are (local sum - the half's total), second-half exponents the local sums themselves.
+    const int pw = warp - 8, ptid = tid - NCH;
+    const int cq = lane & 7, tg = lane >> 3;
+    const int c0 = pw * 32 + cq * 4;
+    PT_DECL
+    // Inputs reach the producer by cp.async, each lane copying exactly the 16-byte vectors of its own tiles INTO
+    // the operand tiles it will overwrite: the raw log-decay of (token t, channels c0..c0+3) lands where Kh[t][c0..]
+    // goes, raw k in the first half of the Kt vector, raw q in the first half of the Qt vector.  A lane only ever
+    // reads what it copied itself, so no barrier is needed, and no register holds data in flight.
+    float beta_next = (n_chunks > 0 && ptid < min(C, n_tok)) ? gb[ptid * b_stride] : 0.f;
+    float gsc_next = (!KDA && n_chunks > 0 && ptid < min(C, n_tok)) ? gg[ptid * g_stride] : 0.f;
+    for (int ch = 0; ch < n_chunks; ++ch) {
+      const uint32_t par = ch & 1;
+      const int t0 = ch * C, ntok = min(C, n_tok - t0);
+      unsigned char *kht_tile = smem + OFF_KHT + par * (128 * 128);
+      // per-token scalars: this chunk's go to their ring slots (the chain warps are at most two chunks behind),
+      // the next chunk's are fetched now and stored one iteration later
+      if (ptid < C) {
+        beta_s[(ch & 3) * C + ptid] = beta_next;
+        if (!KDA) gsc_s[(ch & 3) * C + ptid] = gsc_next;
+        const bool v1 = ch + 1 < n_chunks && ptid < min(C, n_tok - t0 - C);
+        beta_next = v1 ? gb[(t0 + C + ptid) * b_stride] : 0.f;
+        if (!KDA) gsc_next = v1 ? gg[(t0 + C + ptid) * g_stride] : 0.f;
+      }
+      // (a) raw log-decay -> Kh tile, free once MMA1 of the previous chunk has completed
+      if (ch > 0) wait_bar(&misc->bar_ap, par ^ 1, misc, err);
+      PT(0);
+      if constexpr (KDA) {
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          const int t = (jj >> 2) * 16 + tg * 4 + (jj & 3);
+          const bool valid = t < ntok;
+          cp_async16_zfill(sbase + OFF_KH + sw128_offset(32, t, c0), gg + (t0 + (valid ? t : 0)) * g_stride + c0, valid);
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      // (b) raw k, q -> Kt/Qt tile, free once MMA2 of the previous chunk has completed; by then the chain warps
+      //     have also left the chunk before that one, whose parity buffers (post, Kh^T) are reused
+      if (ch > 0) wait_bar(&misc->bar_ro, par ^ 1, misc, err);
+      PT(1);
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) {
+        const int t = (jj >> 2) * 16 + tg * 4 + (jj & 3);
+        const bool valid = t < ntok;
+        const int64_t tt = t0 + (valid ? t : 0);
+        cp_async8_zfill(sbase + OFF_KQ + sw128_offset(64, t, c0), gk + tt * qk_stride + c0, valid);
+        if (WITH_O) cp_async8_zfill(sbase + OFF_KQ + sw128_offset(64, 32 + t, c0), gq + tt * qk_stride + c0, valid);
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      PT(6);
+      if (!KDA) __syncwarp();  // warp 8 wrote gsc_s; the other producer warps meet it at the barrier below
+      if (!KDA) asm volatile("bar.sync 2, 128;" ::: "memory");
+      PT(7);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");  // the log-decay has landed
+      PT(2);
+      // sums: this lane's total, the prefix over the four token groups of the warp (lanes 8 apart), the half's total
+      float run0[2][4], refL[4];
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        float own[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int t = half * 16 + tg * 4 + j;
+          if constexpr (KDA) {
+            const float4 g4 = *reinterpret_cast<const float4 *>(smem + OFF_KH + sw128_offset(32, t, c0));
+            own[0] += g4.x; own[1] += g4.y; own[2] += g4.z; own[3] += g4.w;
+          } else {
+            const float gs = gsc_s[(ch & 3) * C + t];
+            own[0] += gs; own[1] += gs; own[2] += gs; own[3] += gs;
+          }
+        }
+        float tot[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float incl = own[i];
+          float x = __shfl_up_sync(0xffffffffu, incl, 8);
+          if (tg >= 1) incl += x;
+          x = __shfl_up_sync(0xffffffffu, incl, 16);
+          if (tg >= 2) incl += x;
+          run0[half][i] = incl - own[i];                      // accumulated before this lane's first token
+          tot[i] = __shfl_sync(0xffffffffu, incl, cq + 24);    // the half's total
+          if (half == 0) refL[i] = -tot[i] * LOG2E;            // minus the midpoint reference, in log2 units
+        }
+        if (half == 0) {
+          // The factor that takes the state from where the previous chunk left it to this chunk's midpoint needs
+          // the first half's sums only: it is handed to the chain warps before the tiles are built.
+          if (tg == 0) {
+            const float4 post_prev = ch > 0 ? *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0)
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+            *reinterpret_cast<float4 *>(fac_s + par * D + c0) =
+                make_float4(ex2f((post_prev.x + tot[0]) * LOG2E), ex2f((post_prev.y + tot[1]) * LOG2E),
+                            ex2f((post_prev.z + tot[2]) * LOG2E), ex2f((post_prev.w + tot[3]) * LOG2E));
+          }
+          mbar_arrive(&misc->rdy_fac[par]);
+        } else if (tg == 0) {
+          *reinterpret_cast<float4 *>(post_s + par * D + c0) = make_float4(tot[0], tot[1], tot[2], tot[3]);  // G_C - G_m
+        }
+      }
+      asm volatile("cp.async.wait_group 0;" ::: "memory");  // k and q have landed
+      PT(3);
+      const uint64_t l2e2 = pack2(LOG2E, LOG2E), comp2 = pack2(kLog2TruncComp, kLog2TruncComp);
+      const uint64_t qs2 = pack2(a.q_scale, a.q_scale);
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+        const int t4 = half * 16 + tg * 4;
+        uint64_t run01 = half == 0 ? pack2(run0[0][0], run0[0][1]) : pack2(run0[1][0], run0[1][1]);
+        uint64_t run23 = half == 0 ? pack2(run0[0][2], run0[0][3]) : pack2(run0[1][2], run0[1][3]);
+        const uint64_t ref01 = half == 0 ? pack2(refL[0], refL[1]) : 0ull, ref23 = half == 0 ? pack2(refL[2], refL[3]) : 0ull;
+        uint32_t kht[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int t = t4 + j;
+          const uint32_t off_k = OFF_KQ + sw128_offset(64, t, c0), off_q = OFF_KQ + sw128_offset(64, 32 + t, c0);
+          const uint32_t off_h = OFF_KH + sw128_offset(32, t, c0);
+          const uint2 kw = *reinterpret_cast<const uint2 *>(smem + off_k);
+          uint64_t g01, g23;
+          if constexpr (KDA) {
+            const float4 g4 = *reinterpret_cast<const float4 *>(smem + off_h);
+            g01 = pack2(g4.x, g4.y);
+            g23 = pack2(g4.z, g4.w);
+          } else {
+            const float gs = gsc_s[(ch & 3) * C + t];
+            g01 = g23 = pack2(gs, gs);
+          }
+          const uint64_t k01 = pack2(bf16lo(kw.x), bf16hi(kw.x)), k23 = pack2(bf16lo(kw.y), bf16hi(kw.y));
+          run01 = add2(run01, g01);
+          run23 = add2(run23, g23);
+          const uint64_t d01 = fma2(run01, l2e2, ref01), d23 = fma2(run23, l2e2, ref23);  // (G_t - G_m) log2(e)
+          float d[4], dc[4];
+          unpack2(d01, d[0], d[1]);
+          unpack2(d23, d[2], d[3]);
+          unpack2(add2(d01, comp2), dc[0], dc[1]);
+          unpack2(add2(d23, comp2), dc[2], dc[3]);
+          const uint64_t e1_01 = pack2(ex2f(dc[0]), ex2f(dc[1])), e1_23 = pack2(ex2f(dc[2]), ex2f(dc[3]));
+          const uint64_t e2_01 = pack2(ex2f(-d[0]), ex2f(-d[1])), e2_23 = pack2(ex2f(-d[2]), ex2f(-d[3]));
+          float kt[4], kh[4];
+          unpack2(mul2(k01, e1_01), kt[0], kt[1]);
+          unpack2(mul2(k23, e1_23), kt[2], kt[3]);
+          unpack2(mul2(k01, e2_01), kh[0], kh[1]);
+          unpack2(mul2(k23, e2_23), kh[2], kh[3]);
+          if (WITH_O) {
+            const uint2 qw = *reinterpret_cast<const uint2 *>(smem + off_q);
+            const uint64_t q01 = pack2(bf16lo(qw.x), bf16hi(qw.x)), q23 = pack2(bf16lo(qw.y), bf16hi(qw.y));
+            float qt[4];
+            unpack2(mul2(q01, mul2(e1_01, qs2)), qt[0], qt[1]);
+            unpack2(mul2(q23, mul2(e1_23, qs2)), qt[2], qt[3]);
+            *reinterpret_cast<uint4 *>(smem + off_q) =
+                make_uint4(tf32_pre(qt[0]), tf32_pre(qt[1]), tf32_pre(qt[2]), tf32_pre(qt[3]));
+          }
+          *reinterpret_cast<uint4 *>(smem + off_k) =
+              make_uint4(tf32_pre(kt[0]), tf32_pre(kt[1]), tf32_pre(kt[2]), tf32_pre(kt[3]));
+#pragma unroll
+          for (int i = 0; i < 4; ++i) kht[i][j] = tf32_pre(kh[i]);
+          *reinterpret_cast<uint4 *>(smem + off_h) = make_uint4(kht[0][j], kht[1][j], kht[2][j], kht[3][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          *reinterpret_cast<uint4 *>(kht_tile + sw128_offset(128, c0 + i, t4)) =
+              make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
+      }
+      PT(4);
+      fence_smem_to_async();
+      mbar_arrive(&misc->rdy_prep);  // -> MMA1
+      PT(5);
+    }
+    PT_DUMP(ptid == 0, 16);
   } else {
-    // =============================== compute warps ===============================
+    // ================================= chain warps =================================
     const int quad = warp & 3, colh = warp >> 2;                           // TMEM lane quadrant, column half
     const uint32_t tlane = tm + (static_cast<uint32_t>(quad * 32) << 16);  // this warp's TMEM lanes
     const int vrow = quad * 32 + lane;                                     // the TMEM lane this thread owns
-    constexpr float LOG2E = 1.4426950408889634f;
-    PT_DECL
 
-    // cp.async stages of one chunk's inputs
-    auto stage_qk = [&](int ch) {
-      const int t0 = ch * C, ntok = min(C, n_tok - t0);
-      for (int i = tid; i < C * 16; i += NC) {
-        const int t = i >> 4, j = i & 15;
-        const bool valid = t < ntok;
-        const int64_t tt = t0 + (valid ? t : 0);
-        if (go)  // no outputs wanted: q is never read
-          cp_async16_zfill(sbase + OFF_RAWQ + t * 256 + j * 16, reinterpret_cast<const char *>(gq + tt * qk_stride) + j * 16, valid);
-        cp_async16_zfill(sbase + OFF_RAWK + t * 256 + j * 16, reinterpret_cast<const char *>(gk + tt * qk_stride) + j * 16, valid);
-      }
-    };
-    auto stage_g = [&](int ch) {
-      const int t0 = ch * C, ntok = min(C, n_tok - t0);
-      if constexpr (KDA) {
-        for (int i = tid; i < C * 32; i += NC) {
-          const int t = i >> 5, j = i & 31;
-          const bool valid = t < ntok;
-          cp_async16_zfill(sbase + OFF_G + t * 512 + j * 16,
-                           reinterpret_cast<const char *>(gg + (t0 + (valid ? t : 0)) * g_stride) + j * 16, valid);
-        }
-      }
-    };
     auto stage_v = [&](int ch) {
       const int t0 = ch * C, ntok = min(C, n_tok - t0);
-      for (int i = tid; i < C * 16; i += NC) {
+      for (int i = tid; i < C * 16; i += NCH) {
         const int t = i >> 4, j = i & 15;
         const bool valid = t < ntok;
         cp_async16_zfill(sbase + OFF_V + t * 256 + j * 16,
                          reinterpret_cast<const char *>(gv + (t0 + (valid ? t : 0)) * v_stride) + j * 16, valid);
       }
     };
-    // per-token scalars of a chunk (beta, and the scalar log-decay of GDN): threads 0-31 / 32-63
-    auto load_scalar = [&](int ch) -> float {
-      const int t0 = ch * C, ntok = min(C, n_tok - t0);
-      if (tid < C) return tid < ntok ? gb[(t0 + tid) * b_stride] : 0.f;
-      if (!KDA && tid < 2 * C) return (tid - C) < ntok ? gg[(t0 + tid - C) * g_stride] : 0.f;
-      return 0.f;
-    };
-    auto store_scalar = [&](int ch, float x) {
-      if (tid < C) beta_s[(ch & 1) * C + tid] = x;
-      else if (!KDA && tid < 2 * C) gsc_s[(ch & 1) * C + tid - C] = x;
-    };
 
     if (n_chunks > 0) {
-      stage_qk(0);
-      stage_g(0);
+      stage_v(0);
       asm volatile("cp.async.commit_group;" ::: "memory");
-      store_scalar(0, load_scalar(0));
-    }
-    post_s[tid] = 0.f;  // [2][128]: nothing owed before the first chunk
-    // the start state goes into TMEM as it is; the first chunk's state pass scales it like any other
-    if (n_chunks > 0) {
+      // the start state goes into TMEM as it is; the first chunk's state pass scales it like any other
 #pragma unroll 1
       for (int c0 = colh * 64; c0 < colh * 64 + 64; c0 += 32) {
         uint32_t s[32];
@@ -363,107 +633,24 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       tmem_st_wait();
     }
 
+    PT_DECL
     for (int ch = 0; ch < n_chunks; ++ch) {
       const uint32_t par = ch & 1;
       const int t0 = ch * C;
       const int ntok = min(C, n_tok - t0);
       const bool more = ch + 1 < n_chunks;
-      const float *beta_c = beta_s + par * C;
+      const float *beta_c = beta_s + (ch & 3) * C;
+      const float *fac_c = fac_s + par * D;
 
-      // ---- (1) this chunk's inputs have landed; the previous chunk's state update is complete ----
+      // ---- (1) the previous chunk's state update is complete; this chunk's factors and tiles are ready ----
       if (ch > 0) wait_bar(&misc->bar_s, par ^ 1, misc, err);
-      tc_fence_after_sync();
-      asm volatile("cp.async.wait_all;" ::: "memory");
-      sync_compute();
-      const float scalar_next = more ? load_scalar(ch + 1) : 0.f;  // in flight during the chunk
       PT(0);
-
-      // ---- (2) prep: warp = (block of 32 channels, half of the tokens); lane = (4 adjacent channels, 4 consecutive
-      //          tokens), a 4 x 4 tile, so that Kh can also be stored transposed.  The midpoint is the end of the
-      //          first half: first-half exponents are (local sum - the half's total), second-half exponents the
-      //          local sums themselves. ----
-      {
-        const int cq = lane & 7, tg = lane >> 3, half = warp >> 2;
-        const int c0 = (warp & 3) * 32 + cq * 4, t4 = half * 16 + tg * 4;
-        // all shared-memory reads of the tile before its first write
-        uint2 kraw[4], qraw[4];
-        float gl[4][4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          kraw[j] = *reinterpret_cast<const uint2 *>(smem + OFF_RAWK + (t4 + j) * 256 + c0 * 2);
-          qraw[j] = go ? *reinterpret_cast<const uint2 *>(smem + OFF_RAWQ + (t4 + j) * 256 + c0 * 2) : make_uint2(0u, 0u);
-          if constexpr (KDA) {
-            const float4 g4 = *reinterpret_cast<const float4 *>(smem + OFF_G + (t4 + j) * 512 + c0 * 4);
-            gl[j][0] = g4.x; gl[j][1] = g4.y; gl[j][2] = g4.z; gl[j][3] = g4.w;
-          } else {
-            const float gs = gsc_s[par * C + t4 + j];
-            gl[j][0] = gs; gl[j][1] = gs; gl[j][2] = gs; gl[j][3] = gs;
-          }
-        }
-        const float4 post_prev = *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0);
-        // this lane's total, the prefix over the four token groups of the warp (lanes 8 apart), the half's total
-        float run[4], refL[4], tot[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          float incl = gl[0][i] + gl[1][i] + gl[2][i] + gl[3][i];
-          const float own = incl;
-          float x = __shfl_up_sync(0xffffffffu, incl, 8);
-          if (tg >= 1) incl += x;
-          x = __shfl_up_sync(0xffffffffu, incl, 16);
-          if (tg >= 2) incl += x;
-          run[i] = incl - own;                               // accumulated before this lane's first token
-          tot[i] = __shfl_sync(0xffffffffu, incl, cq + 24);   // the half's total
-          refL[i] = half == 0 ? tot[i] * LOG2E : 0.f;
-        }
-        if (tg == 0) {
-          if (half == 0)
-            *reinterpret_cast<float4 *>(fac_s + c0) =
-                make_float4(ex2f((post_prev.x + tot[0]) * LOG2E), ex2f((post_prev.y + tot[1]) * LOG2E),
-                            ex2f((post_prev.z + tot[2]) * LOG2E), ex2f((post_prev.w + tot[3]) * LOG2E));
-          else
-            *reinterpret_cast<float4 *>(post_s + par * D + c0) = make_float4(tot[0], tot[1], tot[2], tot[3]);  // G_C - G_m
-        }
-        uint32_t kht[4][4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int t = t4 + j;
-          const uint2 kw = kraw[j], qw = qraw[j];
-          const float kf[4] = {bf16lo(kw.x), bf16hi(kw.x), bf16lo(kw.y), bf16hi(kw.y)};
-          const float qf[4] = {bf16lo(qw.x), bf16hi(qw.x), bf16lo(qw.y), bf16hi(qw.y)};
-          uint32_t kt[4], qt[4], kh[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            run[i] += gl[j][i];
-            const float d = fmaf(run[i], LOG2E, -refL[i]);      // (G_t - G_m) log2(e)
-            const float e1 = ex2f(d + kLog2TruncComp), e2 = ex2f(-d);
-            kt[i] = tf32_pre(kf[i] * e1);
-            qt[i] = tf32_pre(qf[i] * a.q_scale * e1);
-            kh[i] = tf32_pre(kf[i] * e2);
-            kht[i][j] = kh[i];
-          }
-          *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, t, c0)) = make_uint4(kt[0], kt[1], kt[2], kt[3]);
-          if (go) *reinterpret_cast<uint4 *>(smem + OFF_KQ + sw128_offset(64, 32 + t, c0)) = make_uint4(qt[0], qt[1], qt[2], qt[3]);
-          *reinterpret_cast<uint4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_uint4(kh[0], kh[1], kh[2], kh[3]);
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          *reinterpret_cast<uint4 *>(smem + OFF_KHT + sw128_offset(128, c0 + i, t4)) =
-              make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
-      }
-      fence_smem_to_async();
-      tc_fence_before_sync();
-      mbar_arrive(&misc->rdy_prep);  // -> MMA1
-      sync_compute();                // fac_s visible; raw q/k/g consumed by everyone
-      stage_v(ch);                   // V of this chunk takes the place of the raw log-decay tile
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      if (more) stage_qk(ch + 1);
-      asm volatile("cp.async.commit_group;" ::: "memory");
+      wait_bar(&misc->rdy_fac[par], (ch >> 1) & 1, misc, err);
+      tc_fence_after_sync();
       PT(1);
 
-      // ---- (3) state pass: thread = (value column v, half of the channels); scale the state to this chunk's midpoint ----
+      // ---- (2) state pass: thread = (value column v, half of the channels); scale the state to this chunk's midpoint ----
       {
-        // kept as a real loop (and every other per-chunk phase as compact as possible): the chunk loop is
-        // executed once per 32 tokens by every warp, so its code size decides the instruction-fetch cost
 #pragma unroll 1
         for (int c0 = colh * 64; c0 < colh * 64 + 64; c0 += 32) {
           uint32_t s[32];
@@ -471,7 +658,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           tmem_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
-            const float4 f = *reinterpret_cast<const float4 *>(fac_s + c0 + j);
+            const float4 f = *reinterpret_cast<const float4 *>(fac_c + c0 + j);
             s[j + 0] = __float_as_uint(__uint_as_float(s[j + 0]) * f.x);
             s[j + 1] = __float_as_uint(__uint_as_float(s[j + 1]) * f.y);
             s[j + 2] = __float_as_uint(__uint_as_float(s[j + 2]) * f.z);
@@ -485,96 +672,36 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       mbar_arrive(&misc->rdy_state);  // -> MMA2
       PT(2);
 
-      // ---- (4) A and P out of TMEM; T = (I + A)^-1, by warp 0 (A) and warp 1 (P) ----
-      wait_bar(&misc->bar_ap, par, misc, err);
-      tc_fence_after_sync();
-      PT(3);
-      if (warp < 2) {
+      // ---- (3) P out of TMEM, by warp 1 (lanes 32-63 are its quadrant); A and T are the triangular warp's ----
+      if (WITH_O && warp == 1) {
+        wait_bar(&misc->bar_ap, par, misc, err);
+        tc_fence_after_sync();
         uint32_t x[32];
         tmem_ld32(tlane + COL_AP, x);
         tmem_ld_wait();
         const int t = lane;
-        if (warp == 0) {
-          // lanes 0-31: row t of A = strict_lower(Kt Kh^T) * beta_t, kept in fp32 for the inverse
-          const float bt = beta_c[t] * kInvTruncComp;
+        // row t of P = lower_incl_diag(Qt Kh^T), straight to its operand tile
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            float4 o;
-            o.x = (j + 0 < t) ? bt * __uint_as_float(x[j + 0]) : 0.f;
-            o.y = (j + 1 < t) ? bt * __uint_as_float(x[j + 1]) : 0.f;
-            o.z = (j + 2 < t) ? bt * __uint_as_float(x[j + 2]) : 0.f;
-            o.w = (j + 3 < t) ? bt * __uint_as_float(x[j + 3]) : 0.f;
-            *reinterpret_cast<float4 *>(Lm + t * LDX + j) = o;
-          }
-          __syncwarp();
-          // diagonal 16x16 blocks: lane (block b, column cc) solves (I + L_bb) x = e_cc by forward substitution
-          {
-            const int b = lane >> 4, cc = lane & 15;
-            const float *Lb = Lm + (b * 16) * LDX + b * 16;
-            float xs[16];
-#pragma unroll
-            for (int rr = 0; rr < 16; ++rr) {
-              float acc0 = (rr == cc) ? 1.f : 0.f, acc1 = 0.f;
-#pragma unroll
-              for (int j = 0; j + 1 < rr; j += 2) {
-                acc0 = fmaf(-Lb[rr * LDX + j], xs[j], acc0);
-                acc1 = fmaf(-Lb[rr * LDX + j + 1], xs[j + 1], acc1);
-              }
-              if (rr & 1) acc0 = fmaf(-Lb[rr * LDX + rr - 1], xs[rr - 1], acc0);
-              xs[rr] = acc0 + acc1;
-            }
-#pragma unroll
-            for (int rr = 0; rr < 16; ++rr) Xm[(b * 16 + rr) * LDX + b * 16 + cc] = xs[rr];
-          }
-          __syncwarp();
-          // off-diagonal block: X_10 = -X_11 (L_10 X_00); the product L_10 X_00 is parked in the unused block (0,1)
-          {
-            float acc[2][4] = {};
-            warp_mm_acc(acc, Lm + 16 * LDX, Xm, lane);
-            warp_mm_store(Xm + 16, acc, 1.f, lane);
-            __syncwarp();
-            float acc2[2][4] = {};
-            warp_mm_acc(acc2, Xm + 16 * LDX + 16, Xm + 16, lane);
-            warp_mm_store(Xm + 16 * LDX, acc2, -1.f, lane);
-          }
-        } else if (go) {
-          // lanes 32-63: row t of P = lower_incl_diag(Qt Kh^T), straight to its operand tile
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            uint4 o;
-            o.x = (j + 0 <= t) ? tf32_pre(__uint_as_float(x[j + 0]) * kInvTruncComp) : 0u;
-            o.y = (j + 1 <= t) ? tf32_pre(__uint_as_float(x[j + 1]) * kInvTruncComp) : 0u;
-            o.z = (j + 2 <= t) ? tf32_pre(__uint_as_float(x[j + 2]) * kInvTruncComp) : 0u;
-            o.w = (j + 3 <= t) ? tf32_pre(__uint_as_float(x[j + 3]) * kInvTruncComp) : 0u;
-            *reinterpret_cast<uint4 *>(smem + OFF_PM + sw128_offset(32, t, j)) = o;
-          }
-        }
-      }
-      sync_compute();
-      PT(4);
-      {
-        // T (lower triangle of X, unit diagonal) -> tf32 operand tile; 4 elements per thread
-        const int t = tid >> 3, i0 = (tid & 7) * 4;
-#pragma unroll
-        for (int j = 0; j < 4; j += 4) {
-          const float4 xv = *reinterpret_cast<const float4 *>(Xm + t * LDX + i0 + j);
+        for (int j = 0; j < 32; j += 4) {
           uint4 o;
-          o.x = (i0 + j + 0 <= t) ? tf32_pre(xv.x) : 0u;
-          o.y = (i0 + j + 1 <= t) ? tf32_pre(xv.y) : 0u;
-          o.z = (i0 + j + 2 <= t) ? tf32_pre(xv.z) : 0u;
-          o.w = (i0 + j + 3 <= t) ? tf32_pre(xv.w) : 0u;
-          *reinterpret_cast<uint4 *>(smem + OFF_TM + sw128_offset(32, t, i0 + j)) = o;
+          o.x = (j + 0 <= t) ? tf32_pre(__uint_as_float(x[j + 0]) * kInvTruncComp) : 0u;
+          o.y = (j + 1 <= t) ? tf32_pre(__uint_as_float(x[j + 1]) * kInvTruncComp) : 0u;
+          o.z = (j + 2 <= t) ? tf32_pre(__uint_as_float(x[j + 2]) * kInvTruncComp) : 0u;
+          o.w = (j + 3 <= t) ? tf32_pre(__uint_as_float(x[j + 3]) * kInvTruncComp) : 0u;
+          *reinterpret_cast<uint4 *>(smem + OFF_PM + sw128_offset(32, t, j)) = o;
         }
+        fence_smem_to_async();
       }
-      fence_smem_to_async();
-      PT(5);
+      PT(3);
+      PT(4);
 
-      // ---- (5) RHS^T = beta (V - R)^T as a tf32 pair: high over R^T, low in the consumed A|P columns ----
+      // ---- (4) RHS^T = beta (V - R)^T as a tf32 pair: high over R^T, low in the consumed A|P columns ----
       wait_bar(&misc->bar_ro, par, misc, err);
       tc_fence_after_sync();
-      asm volatile("cp.async.wait_group 1;" ::: "memory");  // V of this chunk (the newer group is the next q, k)
-      sync_compute();
-      PT(6);
+      asm volatile("cp.async.wait_all;" ::: "memory");  // V of this chunk
+      wait_bar(&misc->a_taken, par, misc, err);         // the A|P columns are about to be overwritten
+      sync_chain();
+      PT(5);
       {
         const int tb = colh * 16;
         uint32_t x[16], lo[16];
@@ -593,15 +720,15 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       }
       tc_fence_before_sync();
       mbar_arrive(&misc->rdy_rhs);  // -> MMA3 (T tile and RHS^T are ready)
-      sync_compute();               // everyone is done with V: the next chunk's log-decay tile may land
-      if (more) stage_g(ch + 1);
+      sync_chain();                 // everyone is done with V: the next chunk's V may land
+      if (more) stage_v(ch + 1);
       asm volatile("cp.async.commit_group;" ::: "memory");
-      PT(7);
+      PT(6);
 
-      // ---- (6) U^T as a tf32 pair: high in place, low over the consumed RHS^T ----
+      // ---- (5) U^T as a tf32 pair: high in place, low over the consumed RHS^T ----
       wait_bar(&misc->bar_u, par, misc, err);
       tc_fence_after_sync();
-      PT(8);
+      PT(7);
       {
         const int tb = colh * 16;
         uint32_t x[16], lo[16];
@@ -619,27 +746,27 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       }
       tc_fence_before_sync();
       mbar_arrive(&misc->rdy_u);  // -> MMA4, MMA5
-      PT(9);
+      PT(8);
 
-      // ---- (7) outputs of this chunk ----
+      // ---- (6) outputs of this chunk ----
       wait_bar(&misc->bar_o, par, misc, err);
       tc_fence_after_sync();
-      PT(10);
-      if (go) {
+      PT(9);
+      if (WITH_O) {
         const int tb = colh * 16;
         uint32_t x[16];
         tmem_ld16(tlane + COL_RO + 32 + tb, x);
         tmem_ld_wait();
         if constexpr (sizeof(OT) == 2) {
-          // through shared memory (the Kt/Qt tile is free now) so that global stores are 16 bytes wide
-          __nv_bfloat16 *Os = reinterpret_cast<__nv_bfloat16 *>(smem + OFF_KQ);
+          // through shared memory (the T and P tiles are free now) so that global stores are 16 bytes wide
+          __nv_bfloat16 *Os = reinterpret_cast<__nv_bfloat16 *>(smem + OFF_TM);
 #pragma unroll
           for (int j = 0; j < 16; ++j) Os[(tb + j) * D + vrow] = __float2bfloat16_rn(__uint_as_float(x[j]));
-          sync_compute();
-          for (int i = tid; i < ntok * 16; i += NC) {
+          sync_chain();
+          for (int i = tid; i < ntok * 16; i += NCH) {
             const int t = i >> 4, j = i & 15;
             *reinterpret_cast<uint4 *>(reinterpret_cast<char *>(go + (t0 + t) * v_stride) + j * 16) =
-                *reinterpret_cast<const uint4 *>(smem + OFF_KQ + t * 256 + j * 16);
+                *reinterpret_cast<const uint4 *>(smem + OFF_TM + t * 256 + j * 16);
           }
         } else {
 #pragma unroll
@@ -647,16 +774,21 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
             if (tb + j < ntok) go[(t0 + tb + j) * v_stride + vrow] = __uint_as_float(x[j]);
         }
       }
-      store_scalar(ch + 1, scalar_next);
       tc_fence_before_sync();
-      sync_compute();  // every thread is done with this chunk's tiles before they are rewritten
-      PT(11);
+      mbar_arrive(&misc->tp_free);  // this thread is done with the T|P|O tile region
+      sync_chain();  // every chain thread is done with this chunk's P and O tiles before they are rewritten
+      PT(10);
     }
+    PT_DUMP(tid == 0, 0);
 
     // ---- final state: the factor still owed, then write back ----
-    if (n_chunks > 0) wait_bar(&misc->bar_s, (n_chunks - 1) & 1, misc, err);
-    if (tid < D) fac_s[tid] = ex2f(post_s[((n_chunks + 1) & 1) * D + tid] * LOG2E);
-    sync_compute();
+    if (n_chunks > 0) {
+      wait_bar(&misc->rdy_prep, (n_chunks - 1) & 1, misc, err);  // the last chunk's post_s
+      wait_bar(&misc->bar_s, (n_chunks - 1) & 1, misc, err);
+    }
+    // fac_s is free: the producer has finished (its last arrival was waited for above)
+    if (tid < D) fac_s[tid] = n_chunks > 0 ? ex2f(post_s[((n_chunks - 1) & 1) * D + tid] * LOG2E) : 1.f;
+    sync_chain();
     tc_fence_after_sync();
     {
       const uint8_t *keep = a.row_keep + static_cast<int64_t>(layer) * a.rows_per_layer + static_cast<int64_t>(h) * D;
@@ -678,12 +810,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         }
       }
     }
-    PT(12);
-    PT_DUMP;
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 8) tmem_dealloc(tm, TMEM_COLS);
+  if (warp == WARP_MMA) tmem_dealloc(tm, TMEM_COLS);
 }
 
 template <bool KDA, typename OT, bool WITH_O>
