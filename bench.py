@@ -230,6 +230,22 @@ def build_plan(c, device):
     return plan, rates, gen
 
 
+def max_over_ranks(values, device):
+    """Replicas only: every rank times its own identical share of the work, and the job's time is the slowest rank's.
+    Element-wise maximum of `values` over the ranks of the default process group (the values themselves when no
+    group is initialised)."""
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job(per_rank_units: float, world: int, ms: float) -> float:
+    """Weak scaling: every rank processes `per_rank_units` in `ms` milliseconds (the maximum over ranks)."""
+    return world * per_rank_units / (ms * 1e-3)
+
+
 def token_bytes_per_head(kda: bool, H_v: int, H_k: int) -> float:
     """Algorithmic bytes per (token, value head): q + k (shared by H_v/H_k value heads) + v bf16, g fp32, beta, o bf16."""
     share = H_k / H_v
@@ -385,10 +401,7 @@ def main():
     t_restore = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
     t_refresh = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
     t_total = events[0][0].elapsed_time(events[-1][3]) / args.steps
-    times = torch.tensor([t_pack, t_restore, t_refresh, t_total], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    t_pack, t_restore, t_refresh, t_total = times.tolist()
+    t_pack, t_restore, t_refresh, t_total = max_over_ranks([t_pack, t_restore, t_refresh, t_total], dev)
 
     # ---- the paper's own load policy (Section 4.2): replay the last W tokens from a zero scratch state, merge the
     #      omitted units, no outputs (state-only fast path).  Same streams, W = the suffix length. ----
@@ -410,10 +423,7 @@ def main():
     ev_w[1].record(stream)
     barrier()
     assert dasc.dasc_refresh_status(ws) == 0
-    t_window = torch.tensor([ev_w[0].elapsed_time(ev_w[1]) / args.steps], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(t_window, op=dist.ReduceOp.MAX)
-    t_window = float(t_window)
+    (t_window,) = max_over_ranks([ev_w[0].elapsed_time(ev_w[1]) / args.steps], dev)
 
     # ---- end-to-end leg: host buffers, copies inside the timed region -------------------------
     e2e = None
@@ -462,10 +472,7 @@ def main():
         barrier()
         t_copy = sum(e[0].elapsed_time(e[1]) for e in evs[1:]) / n_steps_e
         t_ref = sum(e[1].elapsed_time(e[2]) for e in evs[1:]) / n_steps_e
-        tt = torch.tensor([t_copy, t_ref], dtype=torch.float64, device=dev)
-        if dist:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t_copy, t_ref = tt.tolist()
+        t_copy, t_ref = max_over_ranks([t_copy, t_ref], dev)
         e_bytes = n_e * (slot * 4 + slot_bytes) + n_e * (slot_bytes + L * dense * 4)
         h2d = h_state.numel() * 4 + (L // ge) * sum(x.numel() * x.element_size() for x in host_streams)
         d2h = h_pool.numel() * h_pool.element_size() + h_out.numel() * 4 + (L // ge) * h_o.numel() * 2
@@ -515,7 +522,7 @@ def main():
     roofline = dict(rl[dominant])
     roofline["kernel"] = dominant
     line = {
-        "metric": "pack_restore_GBps", "value": world * (pack_bytes + restore_bytes) / ((t_pack + t_restore) * 1e-3) / 1e9,
+        "metric": "pack_restore_GBps", "value": whole_job(pack_bytes + restore_bytes, world, t_pack + t_restore) / 1e9,
         "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_total,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(c), "kind": c["kind"], "layers": L, "v_heads": H_v, "k_heads": H_k, "d_k": D,
