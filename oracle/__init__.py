@@ -134,6 +134,15 @@ def slot_budget(budget_bytes, temporal_bytes_per_rank, conv_bytes) -> int:
                                         C.c_int64(conv_bytes)))
 
 
+def tp_balance(units_per_rank):
+    """Section 4.3: (C, send[T][T]) for the store-time redistribution of packed units over the TP group."""
+    U = np.ascontiguousarray(units_per_rank, np.int64)
+    send = np.zeros((U.size, U.size), np.int64)
+    lib().oracle_tp_balance.restype = C.c_int64
+    c = lib().oracle_tp_balance(_p(U), C.c_int32(U.size), _p(send))
+    return int(c), send
+
+
 def _words(a):
     assert a.dtype.itemsize == 4 and a.flags.c_contiguous
     return a.view(np.uint32)

@@ -259,6 +259,25 @@ int64_t oracle_slot_budget(int64_t budget_bytes, const int64_t *temporal_bytes_p
     return budget_bytes / worst - 1;
 }
 
+/* Section 4.3, second stage: the TP group as one storage pool.  With U_r packed
+ * units on rank r and T ranks, the per-rank slot width is C = ceil(sum_r U_r / T).
+ * The paper fixes C and that only remotely owned units move; which unit goes where
+ * is this build's reading: the packed units of all ranks, in rank order, form one
+ * sequence, and the unit at global position p is stored on rank p / C.
+ * send[r*T + s] = number of rank r's units stored on rank s (the diagonal stays put).
+ * Done unit by unit. */
+int64_t oracle_tp_balance(const int64_t *U, int32_t T, int64_t *send)
+{
+    int64_t total = 0;
+    for (int32_t r = 0; r < T; ++r) total += U[r];
+    int64_t C = (total + T - 1) / T;
+    for (int32_t i = 0; i < T * T; ++i) send[i] = 0;
+    int64_t p = 0; /* global position */
+    for (int32_t r = 0; r < T; ++r)
+        for (int64_t u = 0; u < U[r]; ++u, ++p) send[r * T + (int32_t)(p / C)] += 1;
+    return C;
+}
+
 /* ------------------------------------------------------------------ */
 /* Store path (Section 4.1, Appendix B ragged layout): pack             */
 /* ------------------------------------------------------------------ */

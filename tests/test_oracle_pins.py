@@ -225,6 +225,32 @@ def test_slot_budget_and_checkpoint_accounting_match_paper():
     assert p.sum_r == 4 and p.C_ckpt_rag == 1.0 and p.C_temp_pad == 1.0
 
 
+def test_tp_balance_slot_width_and_split_counts():
+    # Section 4.3: C = ceil(sum U_r / T); only remotely owned units move; nothing is lost or duplicated.
+    c, send = oracle.tp_balance([10, 2, 0, 4])
+    assert c == 4                                               # ceil(16 / 4)
+    # hand count: global sequence = 10 units of rank 0, 2 of rank 1, 4 of rank 3; chunks of 4 go to ranks 0..3
+    np.testing.assert_array_equal(send, [[4, 4, 2, 0], [0, 0, 2, 0], [0, 0, 0, 0], [0, 0, 0, 4]])
+    rng = np.random.default_rng(17)
+    for T in (1, 2, 3, 8):
+        for _ in range(20):
+            U = rng.integers(0, 50, size=T)
+            c, send = oracle.tp_balance(U)
+            assert c == -(-int(U.sum()) // T)
+            np.testing.assert_array_equal(send.sum(1), U)       # every unit is sent (or kept) exactly once
+            assert np.all(send.sum(0) <= c)                     # no rank stores more than the slot width
+            assert int(send.sum(0).max()) == min(c, int(U.sum()))  # the bottleneck is the slot width, not max U_r
+            # closed form of the interval overlap: units of rank r occupy [P_r, P_r + U_r), rank s stores [sC, sC + C)
+            P = np.concatenate([[0], np.cumsum(U)])
+            for r in range(T):
+                for s in range(T):
+                    lo, hi = max(P[r], s * c), min(P[r + 1], (s + 1) * c)
+                    assert send[r, s] == max(0, hi - lo)
+    # already balanced payloads: nothing moves
+    c, send = oracle.tp_balance([7, 7, 7])
+    assert c == 7 and np.array_equal(send, 7 * np.eye(3, dtype=np.int64))
+
+
 # ----------------------------------------------------------------------------
 # pack / restore invariants
 # ----------------------------------------------------------------------------
