@@ -225,6 +225,25 @@ dasc_status_t dasc_slot_budget(int64_t budget_bytes, const int64_t *temporal_byt
                                int32_t n_ranks, int64_t conv_bytes, int64_t *out);
 
 /*
+ * TP-balanced placement, second stage (Section 4.3), host arithmetic only: the TP
+ * group is one storage pool with per-rank slot width C = ceil(sum_r U_r / T), U_r
+ * the packed units of one checkpoint on rank r.  The packed units of all ranks,
+ * taken in rank order, form one sequence, and the unit at global position p is
+ * stored on rank p / C (the paper fixes C and that only remotely owned units move;
+ * the assignment is this library's reading).
+ *   units_per_rank  HOST int64[n_ranks]
+ *   slot_width      HOST out: C
+ *   send_counts     HOST out int64[n_ranks][n_ranks]: row r = how many of rank r's
+ *                   units each rank stores, consecutive runs in rank order (the split
+ *                   sizes of the variable-split all-to-all at Store; its transpose
+ *                   is the Load transfer).  The diagonal entry stays on its rank.
+ * The exchange itself is not part of this library's device path (one GPU, no
+ * collective); the Python package carries a torch.distributed form of it.
+ */
+dasc_status_t dasc_tp_balance(const int64_t *units_per_rank, int32_t n_ranks, int64_t *slot_width,
+                              int64_t *send_counts);
+
+/*
  * INT8 checkpoint codec fused into the Store / Load copies (Appendix D, Eq. 10).
  * A row is the d_v values of one (layer, head, key channel) tuple; rows are the
  * plan's retained rows in ragged order (a retained GDN head contributes its d_k

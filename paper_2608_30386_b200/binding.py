@@ -31,6 +31,7 @@ EXPORTS = (
     "dasc_plan_window", "dasc_plan_layer_counts", "dasc_plan_layer_offsets", "dasc_pack", "dasc_restore",
     "dasc_int8_slot_bytes", "dasc_pack_int8", "dasc_restore_int8",
     "dasc_padded_pool_floats", "dasc_pack_padded", "dasc_restore_padded", "dasc_checkpoint_bytes", "dasc_slot_budget",
+    "dasc_tp_balance",
     "dasc_refresh_workspace_bytes", "dasc_refresh", "dasc_refresh_status", "dasc_refresh_window", "dasc_refresh_static",
     "dasc_status_string", "dasc_version",
 )
@@ -96,6 +97,7 @@ def lib() -> C.CDLL:
         L.dasc_restore_padded.argtypes = L.dasc_restore.argtypes
         L.dasc_checkpoint_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_int64)]
         L.dasc_slot_budget.argtypes = [C.c_int64, C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_int64)]
+        L.dasc_tp_balance.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.c_void_p]
         L.dasc_int8_slot_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
         L.dasc_pack_int8.argtypes = L.dasc_pack.argtypes
         L.dasc_restore_int8.argtypes = L.dasc_restore.argtypes
@@ -272,6 +274,16 @@ def dasc_slot_budget(budget_bytes: int, temporal_bytes_per_rank, conv_bytes: int
     _check(lib().dasc_slot_budget(int(budget_bytes), arr.ctypes.data_as(C.c_void_p), int(arr.size), int(conv_bytes),
                                   C.byref(out)), "dasc_slot_budget")
     return int(out.value)
+
+
+def dasc_tp_balance(units_per_rank):
+    """Section 4.3: (C, send[T][T]) — slot width and the split sizes of the store-time all-to-all."""
+    U = np.ascontiguousarray(units_per_rank, np.int64)
+    send = np.zeros((U.size, U.size), np.int64)
+    width = C.c_int64()
+    _check(lib().dasc_tp_balance(U.ctypes.data_as(C.c_void_p), int(U.size), C.byref(width),
+                                 send.ctypes.data_as(C.c_void_p)), "dasc_tp_balance")
+    return int(width.value), send
 
 
 def dasc_int8_slot_bytes(plan: Plan) -> int:

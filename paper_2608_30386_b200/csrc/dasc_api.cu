@@ -234,6 +234,30 @@ dasc_status_t dasc_slot_budget(int64_t budget_bytes, const int64_t *temporal_byt
   return DASC_OK;
 }
 
+dasc_status_t dasc_tp_balance(const int64_t *units_per_rank, int32_t n_ranks, int64_t *slot_width,
+                              int64_t *send_counts) {
+  if (!units_per_rank || !slot_width || !send_counts || n_ranks <= 0) return DASC_ERR_INVALID_ARG;
+  int64_t total = 0;
+  for (int32_t r = 0; r < n_ranks; ++r) {
+    if (units_per_rank[r] < 0) return DASC_ERR_INVALID_ARG;
+    total += units_per_rank[r];
+  }
+  const int64_t width = (total + n_ranks - 1) / n_ranks;
+  *slot_width = width;
+  // rank r's units occupy global positions [begin, begin + U_r); rank s stores positions [s*width, (s+1)*width)
+  int64_t begin = 0;
+  for (int32_t r = 0; r < n_ranks; ++r) {
+    const int64_t end = begin + units_per_rank[r];
+    for (int32_t s = 0; s < n_ranks; ++s) {
+      const int64_t lo = begin > s * width ? begin : s * width;
+      const int64_t hi = end < (s + 1) * width ? end : (s + 1) * width;
+      send_counts[static_cast<int64_t>(r) * n_ranks + s] = hi > lo ? hi - lo : 0;
+    }
+    begin = end;
+  }
+  return DASC_OK;
+}
+
 static int64_t int8_slot_bytes(const dasc_plan_t *plan) {
   const int64_t raw = plan->packed_rows * (plan->info.d_v + 4);
   return (raw + 15) / 16 * 16;

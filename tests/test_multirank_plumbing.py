@@ -57,3 +57,56 @@ def test_reference_arm_runs_on_rank_zero_only():
                        env=env, capture_output=True, text=True, timeout=240)
     assert p.returncode == 0, p.stderr[-2000:]
     assert p.stdout.strip() == ""
+
+
+TP_WORKER = textwrap.dedent("""
+    import json, os, sys
+    sys.path.insert(0, {root!r})
+    import numpy as np, torch, torch.distributed as dist
+    import oracle
+    from paper_2608_30386_b200 import tp_exchange
+    from paper_2608_30386_b200.binding import dasc_tp_balance
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    U = {units!r}
+    width, send = dasc_tp_balance(U)
+    o_width, o_send = oracle.tp_balance(U)
+    assert width == o_width and np.array_equal(send, o_send)
+    # row i of rank r carries the value 1000 * r + i in every column: the global sequence is then recognisable
+    mine = (1000.0 * rank + torch.arange(U[rank], dtype=torch.float32)).unsqueeze(1).repeat(1, 4)
+    assert tp_exchange.gather_unit_counts(U[rank]) == U
+    stored = tp_exchange.store_exchange(mine, U)
+    seq = np.concatenate([1000.0 * r + np.arange(U[r]) for r in range(world)])
+    want = seq[rank * width: (rank + 1) * width]                  # rank s stores global positions [sC, sC + C)
+    assert stored.shape == (len(want), 4) and np.array_equal(stored[:, 0].numpy(), want), (stored[:, 0], want)
+    assert stored.shape[0] <= width
+    back = tp_exchange.load_exchange(stored, U)
+    assert torch.equal(back, mine)                                 # Load is the exact inverse
+    dist.barrier()
+    print("RESULT ok", flush=True)
+    dist.destroy_process_group()
+""")
+
+
+def _run_ranks(script, world):
+    port = _free_port()
+    procs = []
+    for rank in range(world):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port),
+                   CUDA_VISIBLE_DEVICES="")
+        procs.append(subprocess.Popen([sys.executable, "-c", script], env=env, stdout=subprocess.PIPE,
+                                      stderr=subprocess.PIPE, text=True))
+    for p in procs:
+        out, err = p.communicate(timeout=300)
+        assert p.returncode == 0, err[-3000:]
+        assert "RESULT ok" in out
+
+
+def test_tp_balanced_store_and_load_exchange_two_ranks():
+    # Section 4.3: an uneven pair (the heavy rank ships its excess), and an empty rank
+    _run_ranks(TP_WORKER.format(root=ROOT, units=[11, 2]), 2)
+    _run_ranks(TP_WORKER.format(root=ROOT, units=[0, 5]), 2)
+
+
+def test_tp_balanced_store_and_load_exchange_three_ranks():
+    _run_ranks(TP_WORKER.format(root=ROOT, units=[10, 1, 4]), 3)
