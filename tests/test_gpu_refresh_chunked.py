@@ -36,6 +36,18 @@ def test_chunked_ragged_suffixes_both_modes(kind, H_k):
         np.testing.assert_array_equal(got_s[:, keep], s0[:, keep])
 
 
+@pytest.mark.parametrize("with_o", [True, False])
+def test_chunk_boundaries_of_the_producer_pipeline(with_o):
+    # one chunk minus / exactly / plus one token, two and three chunks around their boundaries, two tokens: the
+    # producer warps run a chunk ahead of the chain, so every count of chunks from 1 to 4 and every tail is a case
+    case = make_refresh_case(27, dasc.KDA, 1, 2, 2, 128, 128, [31, 32, 33, 63, 64, 65, 96, 97, 2], scope=dasc.SCOPE_LAYER,
+                             keep_ratio=0.38)
+    ref_s, ref_o = run_refresh_oracle(case, want_o=with_o)
+    got_s, got_o = run_refresh_gpu(case, algo=dasc.ALGO_CHUNKED, want_o=with_o)
+    worst = assert_refresh_close(case, got_s, got_o, ref_s, ref_o, TOL)
+    print("worst rel err", worst)
+
+
 def test_chunked_long_suffix_from_partially_restored_state():
     # aggressive KDA: keep 20 % of the channels, zero-fill the rest, then a 1024-token suffix
     case = make_refresh_case(3, dasc.KDA, 1, 2, 2, 128, 128, [1024], scope=dasc.SCOPE_LAYER, keep_ratio=0.2)
