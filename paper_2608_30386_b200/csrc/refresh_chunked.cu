@@ -74,6 +74,8 @@ constexpr float kTruncComp = 1.000352f;
 constexpr float kInvTruncComp = 1.0f / kTruncComp;
 constexpr float kLog2TruncComp = 5.0774e-4f;  // log2(kTruncComp)
 
+// Development aid, compiled out by default: per-phase cycle counters of the middle CTA (chain thread 0 in slots
+// 0-10, producer thread 0 in slots 16-23), written behind the time-out flag; such a build needs 512 bytes of workspace.
 #ifdef DASC_PHASE_TIMING
 #define PT_DECL long long pt_acc[16] = {0}; long long pt_last = clock64();
 #define PT(i) do { long long pt_now = clock64(); pt_acc[i] += pt_now - pt_last; pt_last = pt_now; } while (0)
@@ -693,7 +695,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         fence_smem_to_async();
       }
       PT(3);
-      PT(4);
 
       // ---- (4) RHS^T = beta (V - R)^T as a tf32 pair: high over R^T, low in the consumed A|P columns ----
       wait_bar(&misc->bar_ro, par, misc, err);
