@@ -121,19 +121,6 @@ __device__ __forceinline__ void cp_async8_zfill(uint32_t smem, const void *gmem,
   asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(smem), "l"(gmem), "r"(n) : "memory");
 }
 
-// non-blocking: has the phase of this parity completed?
-__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -287,22 +274,18 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 
   if (warp == WARP_MMA) {
     // =========================== tensor-core issue warp ===========================
-    // MMA1: [Kt;Qt] Kh^T.  M is padded to 128: rows 64-127 of the A tile are whatever follows it in
-    // shared memory, and land in TMEM lanes 64-127 that nobody reads.
-    auto issue_mma1 = [&]() {
-      tc_fence_after_sync();
-#pragma unroll 1
-      for (int kk = 0; kk < 16; ++kk)  // K = 128 in slices of 8: block kk / 4, 32 bytes per slice inside a block
-        mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
-               desc_kmajor(sbase + OFF_KH + (kk >> 2) * (32 * 128) + (kk & 3) * 32), ID_N32, kk != 0);
-      mma_commit(&misc->bar_ap);
-    };
-    bool ahead = false;  // lane 0: MMA1 of this chunk went out during the previous one
     for (int ch = 0; ch < n_chunks; ++ch) {
       const uint32_t par = ch & 1;
-      if (lane == 0 && !ahead) {
+      // MMA1: [Kt;Qt] Kh^T.  M is padded to 128: rows 64-127 of the A tile are whatever follows it in
+      // shared memory, and land in TMEM lanes 64-127 that nobody reads.
+      if (lane == 0) {
         wait_bar(&misc->rdy_prep, par, misc, err);
-        issue_mma1();
+        tc_fence_after_sync();
+#pragma unroll 1
+        for (int kk = 0; kk < 16; ++kk)  // K = 128 in slices of 8: block kk / 4, 32 bytes per slice inside a block
+          mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
+                 desc_kmajor(sbase + OFF_KH + (kk >> 2) * (32 * 128) + (kk & 3) * 32), ID_N32, kk != 0);
+        mma_commit(&misc->bar_ap);
       }
       __syncwarp();
       // MMA2: S'^T [Kt;Qt]^T, the fp32 state read as a tf32 operand
@@ -329,10 +312,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           mma_ts(tm + COL_U, tm + (kk < 4 ? COL_RO : COL_AP) + (kk & 3) * 8, desc_kmajor(sbase + OFF_TM + (kk & 3) * 32),
                  ID_N32, kk != 0);
         mma_commit(&misc->bar_u);
-        // The A|P columns are free again (MMA3 was their last reader, and the tensor pipe runs in order): if the
-        // next chunk's tiles are ready, its MMA1 goes out now instead of behind this chunk's state update.
-        ahead = ch + 1 < n_chunks && !misc->abort_flag && mbar_test_wait(&misc->rdy_prep, par ^ 1);
-        if (ahead) issue_mma1();
       }
       // MMA4: O^T += U^T P^T (high part of U);  MMA5: S'^T += U^T Kh (U as a pair: high in place, low over RHS^T)
       if (lane == 0) wait_bar(&misc->rdy_u, par, misc, err);
