@@ -224,7 +224,21 @@ def build_plan(c, device):
     rates = synth.skew_layers(synth.decay_rates(gen, c["L"], c["H_v"], D if kda else 1, c["rate_lo"], 1.0),
                               c.get("layer_skew", 0.0))
     A_log, dt = synth.decay_params(rates)
-    plan = dasc.dasc_plan(dasc.KDA if kda else dasc.GDN, c["L"], c["H_v"], c["H_k"], D, D, A_log.numpy(), dt.numpy(),
+    kind = dasc.KDA if kda else dasc.GDN
+    if c.get("mixed_heads") and kda:
+        # Every head draws its own keep ratio from the sweep's set, so the per-head channel counts are ragged by
+        # construction.  The selection itself stays in the library: one head-scope plan per ratio (host only), and each
+        # head takes the mask of the plan with its ratio; the union goes in as an explicit mask.
+        ratios = (0.25, 0.38, 0.5, 1.0)
+        masks = [dasc.dasc_plan(kind, c["L"], c["H_v"], c["H_k"], D, D, A_log.numpy(), dt.numpy(), sel=dasc.SEL_TOP_RATIO,
+                                scope=dasc.SCOPE_HEAD, keep_ratio=r, device=-1).mask().reshape(c["L"], c["H_v"], D)
+                 for r in ratios]
+        pick = torch.randint(0, len(ratios), (c["L"], c["H_v"]), generator=gen).numpy()
+        mask = np.choose(pick[:, :, None], masks)
+        plan = dasc.dasc_plan(kind, c["L"], c["H_v"], c["H_k"], D, D, A_log.numpy(), dt.numpy(), sel=dasc.SEL_EXPLICIT,
+                              explicit_mask=mask.reshape(c["L"], -1), device=device)
+        return plan, rates, gen
+    plan = dasc.dasc_plan(kind, c["L"], c["H_v"], c["H_k"], D, D, A_log.numpy(), dt.numpy(),
                           sel=dasc.SEL_TOP_RATIO, scope=dasc.SCOPE_MODEL if c.get("scope") == "model" else dasc.SCOPE_LAYER,
                           keep_ratio=c["keep"], device=device)
     return plan, rates, gen
@@ -270,6 +284,8 @@ def main():
                     help="checkpoint pool layout (Appendix B): ragged [slots][sum r_l] or padded [L][slots][R_max]")
     ap.add_argument("--scope", default="layer", choices=["layer", "model"],
                     help="selection scope of the keep ratio; 'model' makes per-layer counts differ (padding appears)")
+    ap.add_argument("--mixed-heads", action="store_true",
+                    help="every head draws its own keep ratio from {0.25, 0.38, 0.5, 1.0} (ragged per-head channel counts)")
     ap.add_argument("--layer-skew", type=float, default=0.0,
                     help="imbalanced per-layer decay profile: layer rates scaled by exp(skew * (l/(L-1) - 1/2))")
     ap.add_argument("--codec", default="fp32", choices=["fp32", "int8"],
@@ -285,6 +301,7 @@ def main():
     c["codec"] = args.codec
     c["scope"] = args.scope
     c["layer_skew"] = args.layer_skew
+    c["mixed_heads"] = args.mixed_heads
     if args.impl == "reference":
         run_reference(args, c)
         return
@@ -507,7 +524,9 @@ def main():
         "refresh": {"bound": "hbm", "achieved": refresh_gbs, "peak": hbm, "unit": "GB/s", "frac": refresh_gbs / hbm,
                     "traffic": None, "peak_source": src, "tflops_min_form": refresh_tflops,
                     "frac_of_fp32_alu": refresh_tflops / alu_tflops, "tflops_tf32_issued": tf32_issued,
-                    "tf32_peak": TF32_OVER_BF16 * tf, "frac_of_tf32_tensor": tf32_issued / (TF32_OVER_BF16 * tf)},
+                    "tf32_peak": TF32_OVER_BF16 * tf, "frac_of_tf32_tensor": tf32_issued / (TF32_OVER_BF16 * tf),
+                    # the token-by-token minimum (7 d_k d_v flop per token-head) against the same tensor peak
+                    "frac_useful_of_tf32_tensor": refresh_tflops / (TF32_OVER_BF16 * tf)},
     }
     if c["name"] == "kda_serving" and not int8:      # the workload the capture was made on
         rl["pack"]["traffic"] = NCU_TRAFFIC_OVER_ALGORITHMIC["pack"] * pack_bytes
@@ -526,7 +545,9 @@ def main():
         "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_total,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": workload_name(c), "kind": c["kind"], "layers": L, "v_heads": H_v, "k_heads": H_k, "d_k": D,
-                   "d_v": D, "requests": N_REQ, "keep_ratio": c["keep"], "codec": args.codec, "layout": args.layout, "selection_scope": args.scope,
+                   "d_v": D, "requests": N_REQ, "keep_ratio": c["keep"], "codec": args.codec, "layout": args.layout,
+                   "selection_scope": "mixed per-head ratios" if args.mixed_heads else args.scope,
+                   "units_retained_fraction": plan.units_retained / plan.units_total,
                    "pool_bytes": pool.numel() * pool.element_size(), "suffix_tokens": SUFFIX, "refresh_algo": args.algo,
                    "stream_layers_resident": group,
                    "l2": "inputs larger than L2 (GiBs of states and token streams per step); no flush needed",
@@ -553,7 +574,7 @@ def main():
     }
     if e2e:
         line["e2e"] = e2e
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline and world == 1 and not args.mixed_heads:  # the oracle leg times the per-layer rule
         line["cpu_baseline"] = {k2: v2 for k2, v2 in oracle_leg(c).items() if k2 != "seconds"}
     print(json.dumps(line))
     if dist:

@@ -150,3 +150,42 @@ def test_serving_scale_kda_sampled_against_oracle(ratio):
         o_out = np.full_like(one, np.float32(-1.0))
         oracle.restore(oplan.mask, d, o_pool, int(plan.slot_floats), [0], o_out, H * d * d, 0, [0])
         np.testing.assert_array_equal(bits(out[:, r]), o_out.view(np.uint32))
+
+
+def test_mixed_per_head_ratios_explicit_mask():
+    """Every head keeps its own fraction of channels (ragged per-head counts): the mask is assembled from head-scope
+    plans of the library and fed back as an explicit mask; pack / restore against the oracle on that mask."""
+    dev = "cuda"
+    gen = synth.generator(9)
+    L, H, d = 3, 8, 128
+    rates = synth.decay_rates(gen, L, H, d, 1e-3, 1.0)
+    A, B = synth.decay_params(rates)
+    ratios = (0.25, 0.38, 0.5, 1.0)
+    masks = [dasc.dasc_plan(dasc.KDA, L, H, H, d, d, A.numpy(), B.numpy(), sel=dasc.SEL_TOP_RATIO, scope=dasc.SCOPE_HEAD,
+                            keep_ratio=r, device=-1).mask().reshape(L, H, d) for r in ratios]
+    pick = torch.randint(0, 4, (L, H), generator=gen).numpy()
+    mask = np.choose(pick[:, :, None], masks).reshape(L, H * d).astype(np.uint8)
+    counts = mask.reshape(L, H, d).sum(-1)
+    assert len(set(counts.ravel().tolist())) > 1                    # ragged per-head channel counts
+    plan = dasc.dasc_plan(dasc.KDA, L, H, H, d, d, A.numpy(), B.numpy(), sel=dasc.SEL_EXPLICIT, explicit_mask=mask)
+    oplan = oracle.plan(oracle.KDA, L, H, d, A.numpy(), B.numpy(), sel=oracle.SEL_EXPLICIT, explicit_mask=mask,
+                        unit_bytes=d * 4)
+    np.testing.assert_array_equal(plan.mask(), oplan.mask)
+    np.testing.assert_array_equal(plan.mask(), mask)
+    dense, n_req = H * d * d, 5
+    state = synth.states(gen, (n_req, L, dense))
+    synth.special_values_(state, gen)
+    ids = torch.arange(n_req, dtype=torch.int32)
+    slots = torch.flip(ids, [0]).contiguous()
+    slot = int(plan.slot_floats)
+    d_pool = torch.full((n_req, slot), 7.0, device=dev)
+    dasc.dasc_pack(plan, state.to(dev), dense, L * dense, ids.to(dev), d_pool, slots.to(dev))
+    d_out = torch.full((n_req, L, dense), -3.0, device=dev)
+    dasc.dasc_restore(plan, d_pool, slots.to(dev), d_out, dense, L * dense, ids.to(dev))
+    torch.cuda.synchronize()
+    o_pool = np.full((n_req, slot), np.float32(7.0))
+    oracle.pack(oplan.mask, d, state.numpy(), dense, L * dense, ids.numpy(), o_pool, slot, slots.numpy())
+    o_out = np.full((n_req, L, dense), np.float32(-3.0))
+    oracle.restore(oplan.mask, d, o_pool, slot, slots.numpy(), o_out, dense, L * dense, ids.numpy())
+    np.testing.assert_array_equal(bits(d_pool), o_pool.view(np.uint32))
+    np.testing.assert_array_equal(bits(d_out), o_out.view(np.uint32))
