@@ -170,3 +170,44 @@ def test_mixed_trace_two_streams():
         worst = check_sampled_refresh(dasc.KDA, plan, oplan, restored, active, ls, rs, q, k, v, g, beta, o, cu, units, TOL)
         print(f"mixed trace wave {w}: {T} tokens, worst sampled rel err {worst:.2e}")
         free_slot += wave
+
+
+def test_kda_serving_config_refresh_in_the_benchmarks_launch():
+    """The benchmark line's own refresh launch: 64 requests x 24 layers x 32 heads in ONE call (49,152 CTAs), keep 0.38
+    per layer, 256-token bf16 suffix, bf16 outputs, plus the state-only window refresh of the same tokens.  Sampled
+    (request, layer, head) units against the oracle on the same bits."""
+    dev = "cuda"
+    L, H, d, n_req, suffix = 24, 32, 128, 64, 256
+    gen = synth.generator(1)
+    rates = synth.decay_rates(gen, L, H, d, 1e-3, 1.0)
+    plan, oplan = make_plans(dasc.KDA, L, H, H, d, d, rates, sel=dasc.SEL_TOP_RATIO, keep_ratio=0.38)
+    dgen = synth.generator(1, dev)
+    dense = H * d * d
+    ls, rs = n_req * dense, dense
+    active = synth.states(dgen, (L, n_req, dense), dev)
+    ids = torch.arange(n_req, dtype=torch.int32, device=dev)
+    T = n_req * suffix
+    cu = synth.uniform_cu_seqlens(n_req, suffix)
+    q, k, v, g, beta = _streams(dgen, synth.KDA, L, T, H, H, d, rates, dev)
+    o = torch.empty((L, T, H, d), dtype=torch.bfloat16, device=dev)
+    ws = torch.zeros(dasc.dasc_refresh_workspace_bytes(plan, n_req, L), dtype=torch.uint8, device=dev)
+    before = active.clone()
+    dasc.dasc_refresh(plan, active, ls, rs, ids, q, k, v, g, beta, cu.to(dev), T, suffix, o=o, workspace=ws)
+    torch.cuda.synchronize()
+    assert dasc.dasc_refresh_status(ws) == 0
+    units = sample_units(11, n_req, L, H, 16)
+    # bf16 outputs carry their own rounding (half an ulp is up to 2^-8 of the value): states at 1e-3, outputs at 1e-3 + 2^-8
+    worst = check_sampled_refresh(dasc.KDA, plan, oplan, before, active, ls, rs, q, k, v, g, beta, None, cu, units, TOL)
+    worst_o = check_sampled_refresh(dasc.KDA, plan, oplan, before, active, ls, rs, q, k, v, g, beta, o, cu, units,
+                                    TOL + 2.0 ** -8)
+    print(f"KDA serving config, one launch: worst sampled state err {worst:.2e}, with bf16 outputs {worst_o:.2e}")
+    # the paper's load policy on the same launch shape: scratch replay of the same 256 tokens, no outputs
+    merged = before.clone()
+    wb = torch.empty(n_req, dtype=torch.int32, device=dev)
+    dasc.dasc_refresh_window(plan, merged, ls, rs, ids, None, k, v, g, beta, cu.to(dev), T, wb, window=suffix, workspace=ws)
+    torch.cuda.synchronize()
+    assert dasc.dasc_refresh_status(ws) == 0
+    assert torch.equal(wb.cpu(), cu[:-1])
+    worst_w = check_sampled_refresh(dasc.KDA, plan, oplan, before, merged, ls, rs, q, k, v, g, beta, None, cu, units, TOL,
+                                    mode=oracle.MODE_SCRATCH_MERGE_LOCAL)
+    print(f"window refresh, state only: worst sampled err {worst_w:.2e}")
