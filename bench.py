@@ -40,8 +40,8 @@ import torch  # noqa: E402
 D = 128
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 TF32_OVER_BF16 = 0.489        # nominal dense 1.1 : 2.25
-CHUNKED_FLOPS_PER_TOKEN_HEAD = 188416   # tf32 flops the chunked kernel issues per (token, head): 32-token chunks,
-                                        # MMA1 padded to M = 128, hi/lo pairs in MMA3 and MMA5
+CHUNKED_FLOPS_PER_TOKEN_HEAD = 196608   # tf32 flops the chunked kernel issues per (token, head): 32-token chunks,
+                                        # MMA1 padded to M = 128, hi/lo pairs in MMA3, MMA4 and MMA5
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes, from one ncu full-set capture of
 # the KDA serving workload at 8 requests and a 128-token suffix (a full-size launch is too large to capture); every

@@ -312,8 +312,20 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           mma_ts(tm + COL_U, tm + (kk < 4 ? COL_RO : COL_AP) + (kk & 3) * 8, desc_kmajor(sbase + OFF_TM + (kk & 3) * 32),
                  ID_N32, kk != 0);
         mma_commit(&misc->bar_u);
+        // U^T stays where MMA3 leaves it: read as an operand, each fp32 value gives its high (truncated) part, and
+        // the chain warps supply the exact remainder afterwards (U = U_hi + U_lo).  The high-part products go out at
+        // once, behind MMA3 in the tensor pipe's issue order, without a round trip through the chain warps:
+        // MMA4 (high): O^T += U_hi^T P^T;  MMA5 (high): S'^T += U_hi^T Kh
+        if (WITH_O) {
+#pragma unroll 1
+          for (int kk = 0; kk < 4; ++kk)
+            mma_ts(tm + COL_RO + 32, tm + COL_U + kk * 8, desc_kmajor(sbase + OFF_PM + kk * 32), ID_N32, true);
+        }
+#pragma unroll 1
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ts(tm + COL_S, tm + COL_U + kk * 8, desc_kmajor(sbase + OFF_KHT + par * (128 * 128) + kk * 32), ID_N128, true);
       }
-      // MMA4: O^T += U^T P^T (high part of U);  MMA5: S'^T += U^T Kh (U as a pair: high in place, low over RHS^T)
+      // MMA4 (low), MMA5 (low): the same with U_lo^T, which the chain warps wrote over the consumed RHS^T
       if (lane == 0) wait_bar(&misc->rdy_u, par, misc, err);
       __syncwarp();
       if (lane == 0) {
@@ -321,13 +333,12 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         if (WITH_O) {
 #pragma unroll 1
           for (int kk = 0; kk < 4; ++kk)
-            mma_ts(tm + COL_RO + 32, tm + COL_U + kk * 8, desc_kmajor(sbase + OFF_PM + kk * 32), ID_N32, true);
+            mma_ts(tm + COL_RO + 32, tm + COL_RO + kk * 8, desc_kmajor(sbase + OFF_PM + kk * 32), ID_N32, true);
         }
         mma_commit(&misc->bar_o);
 #pragma unroll 1
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tm + COL_S, tm + (kk < 4 ? COL_U : COL_RO) + (kk & 3) * 8,
-                 desc_kmajor(sbase + OFF_KHT + par * (128 * 128) + (kk & 3) * 32), ID_N128, true);
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ts(tm + COL_S, tm + COL_RO + kk * 8, desc_kmajor(sbase + OFF_KHT + par * (128 * 128) + kk * 32), ID_N128, true);
         mma_commit(&misc->bar_s);
       }
       __syncwarp();
@@ -705,23 +716,20 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       asm volatile("cp.async.commit_group;" ::: "memory");
       PT(6);
 
-      // ---- (5) U^T as a tf32 pair: high in place, low over the consumed RHS^T ----
+      // ---- (5) the part of U^T the tensor core drops when it reads it (the low 13 mantissa bits), written over
+      //          the consumed RHS^T: U = U_hi + U_lo exactly ----
       wait_bar(&misc->bar_u, par, misc, err);
       tc_fence_after_sync();
       PT(7);
       {
         const int tb = colh * 16;
-        uint32_t x[16], lo[16];
+        uint32_t x[16];
         tmem_ld16(tlane + COL_U + tb, x);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float u = __uint_as_float(x[j]);
-          x[j] = to_tf32(u);
-          lo[j] = tf32_pre(u - __uint_as_float(x[j]));
-        }
-        tmem_st16(tlane + COL_U + tb, x);
-        tmem_st16(tlane + COL_RO + tb, lo);
+        for (int j = 0; j < 16; ++j)
+          x[j] = tf32_pre(__uint_as_float(x[j]) - __uint_as_float(x[j] & 0xFFFFE000u));
+        tmem_st16(tlane + COL_RO + tb, x);
         tmem_st_wait();
       }
       tc_fence_before_sync();
