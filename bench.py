@@ -269,7 +269,7 @@ def token_bytes_per_head(kda: bool, H_v: int, H_k: int) -> float:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="dasc", choices=["dasc", "reference"])
     ap.add_argument("--algo", default="auto", choices=["auto", "sequential", "chunked"])
