@@ -33,33 +33,41 @@ __device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) {
                : "memory");
 }
 
-// grid = (ceil(packed_vecs / (kThreads*UNROLL)), pairs).  A "vec" is 16 bytes of a row.
+// grid = (ceil(R_max * vecs_per_unit / (kThreads*UNROLL)), n_layers, pairs).  A "vec" is 16 bytes of a row.  One
+// layer per block row: the layer's first packed row and its count are per-block constants, the source address
+// needs the dense row only, and a block past its layer's count leaves at once.
 template <int UNROLL>
-__global__ void __launch_bounds__(kThreads) pack_kernel(const uint4 *__restrict__ state, int64_t layer_stride4,
-                                                        int64_t req_stride4, const int32_t *__restrict__ src_req,
-                                                        uint4 *__restrict__ pool, int64_t slot_stride4,
-                                                        const int32_t *__restrict__ dst_slot,
-                                                        const DascRowSrc *__restrict__ row_src, uint32_t packed_vecs,
-                                                        uint32_t vecs_per_row, int32_t n_pairs) {
+__global__ void __launch_bounds__(kThreads, 8) pack_kernel(const uint4 *__restrict__ state, int64_t layer_stride4,
+                                                           int64_t req_stride4, const int32_t *__restrict__ src_req,
+                                                           uint4 *__restrict__ pool, int64_t slot_stride4,
+                                                           const int32_t *__restrict__ dst_slot,
+                                                           const DascRowSrc *__restrict__ row_src,
+                                                           const int32_t *__restrict__ layer_row_off,
+                                                           uint32_t vecs_per_row, int32_t n_pairs) {
   const uint32_t base = blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
-  for (int32_t pair = blockIdx.y; pair < n_pairs; pair += gridDim.y) {
-    const uint4 *src_base = state + static_cast<int64_t>(__ldg(src_req + pair)) * req_stride4;
-    uint4 *dst_base = pool + static_cast<int64_t>(__ldg(dst_slot + pair)) * slot_stride4;
+  const int32_t layer = blockIdx.y;
+  const uint32_t first = static_cast<uint32_t>(__ldg(layer_row_off + layer));
+  const uint32_t layer_vecs = (static_cast<uint32_t>(__ldg(layer_row_off + layer + 1)) - first) * vecs_per_row;
+  if (blockIdx.x * (kThreads * UNROLL) >= layer_vecs) return;
+  const int2 *src_l = reinterpret_cast<const int2 *>(row_src) + first;  // {layer, dense row} of the layer's packed rows
+  for (int32_t pair = blockIdx.z; pair < n_pairs; pair += gridDim.z) {
+    const uint4 *src_base = state + static_cast<int64_t>(__ldg(src_req + pair)) * req_stride4 + layer * layer_stride4;
+    uint4 *dst_base = pool + static_cast<int64_t>(__ldg(dst_slot + pair)) * slot_stride4 +
+                      static_cast<int64_t>(first) * vecs_per_row;
     uint4 val[UNROLL];
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
       const uint32_t i = base + u * kThreads;
-      if (i < packed_vecs) {
+      if (i < layer_vecs) {
         const uint32_t row = i / vecs_per_row;
         const uint32_t vec = i - row * vecs_per_row;
-        const int2 s = __ldg(reinterpret_cast<const int2 *>(row_src) + row);  // {layer, dense row}
-        val[u] = ld_stream(src_base + s.x * layer_stride4 + static_cast<int64_t>(s.y) * vecs_per_row + vec);
+        val[u] = ld_stream(src_base + static_cast<int64_t>(__ldg(src_l + row).y) * vecs_per_row + vec);
       }
     }
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
       const uint32_t i = base + u * kThreads;
-      if (i < packed_vecs) st_stream(dst_base + i, val[u]);
+      if (i < layer_vecs) st_stream(dst_base + i, val[u]);
     }
   }
 }
@@ -111,12 +119,12 @@ int dasc_launch_pack(const dasc_plan_s *plan, const float *state, int64_t layer_
   const uint64_t packed_vecs = static_cast<uint64_t>(plan->packed_rows) * vpr;
   if (packed_vecs == 0 || n_pairs == 0) return cudaSuccess;
   const uint32_t per_block = kThreads * kPackUnroll;
-  dim3 grid(static_cast<uint32_t>((packed_vecs + per_block - 1) / per_block),
-            static_cast<uint32_t>(n_pairs < 65535 ? n_pairs : 65535));
+  const uint64_t max_layer_vecs = static_cast<uint64_t>(plan->info.r_max) * (plan->info.unit_floats / 4);
+  dim3 grid(static_cast<uint32_t>((max_layer_vecs + per_block - 1) / per_block),
+            static_cast<uint32_t>(plan->info.n_layers), static_cast<uint32_t>(n_pairs < 65535 ? n_pairs : 65535));
   pack_kernel<kPackUnroll><<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
       reinterpret_cast<const uint4 *>(state), layer_stride / 4, req_stride / 4, src_req,
-      reinterpret_cast<uint4 *>(pool), slot_stride / 4, dst_slot, plan->d_row_src,
-      static_cast<uint32_t>(packed_vecs), vpr, n_pairs);
+      reinterpret_cast<uint4 *>(pool), slot_stride / 4, dst_slot, plan->d_row_src, plan->d_layer_row_off, vpr, n_pairs);
   return static_cast<int>(cudaGetLastError());
 }
 

@@ -25,38 +25,40 @@ __device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) {
                : "memory");
 }
 
-// grid = (ceil(packed_vecs / (kThreads*kUnroll)), pairs).  entry_stride4 = 16-byte vectors between
-// consecutive (layer, slot) blocks of the pool: R_max rows of vecs_per_row vectors.
+// grid = (ceil(R_max * vecs_per_unit / (kThreads*kUnroll)), n_layers, pairs): one layer per block row, so the layer's
+// first packed row is a per-block constant and no load depends on another table.  entry_stride4 = 16-byte vectors
+// between consecutive (layer, slot) blocks of the pool: R_max rows of vecs_per_row vectors.
 __global__ void __launch_bounds__(kThreads, 8) pack_padded_kernel(const uint4 *__restrict__ state, int64_t layer_stride4,
                                                                int64_t req_stride4, const int32_t *__restrict__ src_req,
                                                                uint4 *__restrict__ pool, int64_t n_slots,
                                                                int64_t entry_stride4, const int32_t *__restrict__ dst_slot,
                                                                const DascRowSrc *__restrict__ row_src,
                                                                const int32_t *__restrict__ layer_row_off,
-                                                               uint32_t packed_vecs, uint32_t vecs_per_row,
-                                                               int32_t n_pairs) {
+                                                               uint32_t vecs_per_row, int32_t n_pairs) {
   const uint32_t base = blockIdx.x * (kThreads * kUnroll) + threadIdx.x;
-  for (int32_t pair = blockIdx.y; pair < n_pairs; pair += gridDim.y) {
-    const uint4 *src_base = state + static_cast<int64_t>(__ldg(src_req + pair)) * req_stride4;
-    const int64_t slot = __ldg(dst_slot + pair);
+  const int32_t layer = blockIdx.y;
+  const uint32_t first = static_cast<uint32_t>(__ldg(layer_row_off + layer));
+  const uint32_t layer_vecs = (static_cast<uint32_t>(__ldg(layer_row_off + layer + 1)) - first) * vecs_per_row;
+  if (blockIdx.x * (kThreads * kUnroll) >= layer_vecs) return;
+  const int2 *src_l = reinterpret_cast<const int2 *>(row_src) + first;  // {layer, dense row} of the layer's packed rows
+  for (int32_t pair = blockIdx.z; pair < n_pairs; pair += gridDim.z) {
+    const uint4 *src_base = state + static_cast<int64_t>(__ldg(src_req + pair)) * req_stride4 + layer * layer_stride4;
+    uint4 *dst_base = pool + (layer * n_slots + __ldg(dst_slot + pair)) * entry_stride4;
     uint4 val[kUnroll];
-    int64_t dst[kUnroll];
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const uint32_t i = base + u * kThreads;
-      dst[u] = -1;
-      if (i < packed_vecs) {
+      if (i < layer_vecs) {
         const uint32_t row = i / vecs_per_row;
         const uint32_t vec = i - row * vecs_per_row;
-        const int2 s = __ldg(reinterpret_cast<const int2 *>(row_src) + row);  // {layer, dense row}
-        val[u] = ld_stream(src_base + s.x * layer_stride4 + static_cast<int64_t>(s.y) * vecs_per_row + vec);
-        const uint32_t row_in_layer = row - static_cast<uint32_t>(__ldg(layer_row_off + s.x));
-        dst[u] = (s.x * n_slots + slot) * entry_stride4 + static_cast<int64_t>(row_in_layer) * vecs_per_row + vec;
+        val[u] = ld_stream(src_base + static_cast<int64_t>(__ldg(src_l + row).y) * vecs_per_row + vec);
       }
     }
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u)
-      if (dst[u] >= 0) st_stream(pool + dst[u], val[u]);
+    for (int u = 0; u < kUnroll; ++u) {
+      const uint32_t i = base + u * kThreads;
+      if (i < layer_vecs) st_stream(dst_base + i, val[u]);
+    }
   }
 }
 
@@ -108,12 +110,12 @@ int dasc_launch_pack_padded(const dasc_plan_s *plan, const float *state, int64_t
   const int64_t rows_per_unit = plan->info.unit_floats / plan->info.d_v;
   const int64_t entry_stride4 = plan->info.r_max * rows_per_unit * vpr;
   const uint32_t per_block = kThreads * kUnroll;
-  dim3 grid(static_cast<uint32_t>((packed_vecs + per_block - 1) / per_block),
-            static_cast<uint32_t>(n_pairs < 65535 ? n_pairs : 65535));
+  const uint64_t max_layer_vecs = static_cast<uint64_t>(entry_stride4);
+  dim3 grid(static_cast<uint32_t>((max_layer_vecs + per_block - 1) / per_block),
+            static_cast<uint32_t>(plan->info.n_layers), static_cast<uint32_t>(n_pairs < 65535 ? n_pairs : 65535));
   pack_padded_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
       reinterpret_cast<const uint4 *>(state), layer_stride / 4, req_stride / 4, src_req, reinterpret_cast<uint4 *>(pool),
-      n_slots, entry_stride4, dst_slot, plan->d_row_src, plan->d_layer_row_off, static_cast<uint32_t>(packed_vecs), vpr,
-      n_pairs);
+      n_slots, entry_stride4, dst_slot, plan->d_row_src, plan->d_layer_row_off, vpr, n_pairs);
   return static_cast<int>(cudaGetLastError());
 }
 
