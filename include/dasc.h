@@ -55,7 +55,8 @@ typedef enum {
   DASC_ERR_ALLOC = 4,       /* host or device allocation failed (dasc_plan only) */
   DASC_ERR_CUDA = 5,        /* a CUDA runtime call or launch failed */
   DASC_ERR_WORKSPACE = 6,   /* workspace missing, misaligned or too small */
-  DASC_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out (reported by dasc_refresh_status) */
+  DASC_ERR_TIMEOUT = 7,     /* a bounded device-side wait ran out (reported by dasc_refresh_status) */
+  DASC_ERR_DOMAIN = 8       /* log-decay outside the chunked kernel's range (reported by dasc_refresh_status) */
 } dasc_status_t;
 
 typedef enum { DASC_KDA = 0, DASC_GDN = 1 } dasc_kind_t;
@@ -307,15 +308,19 @@ dasc_status_t dasc_restore_int8(const dasc_plan_t *plan, const void *pool_base,
  *   and, for every 16 consecutive tokens and every channel, sum |g| <= 80
  *   (decay factors are formed relative to the chunk midpoint in fp32); it
  *   returns DASC_ERR_SHAPE otherwise.  AUTO picks CHUNKED when shape
- *   and dtype allow it and SEQUENTIAL when they do not; the bound on g is
- *   the caller's to know.
+ *   and dtype allow it and SEQUENTIAL when they do not.  The bound on g is
+ *   checked on the device, per channel and half chunk, while the decay sums
+ *   are formed: a violation is recorded in the workspace (DASC_ERR_DOMAIN
+ *   from dasc_refresh_status) and the states and outputs of that call are
+ *   unspecified (possibly inf or NaN); rerun it with DASC_ALGO_SEQUENTIAL.
  *
  * workspace: DEVICE scratch of at least dasc_refresh_workspace_bytes(), 256-byte
  *   aligned, private to this call until it completes; may be NULL when that
  *   size is 0.
  * Errors: bad arguments -> no launch.  A bounded device-side wait that runs
- *   out sets a flag in the workspace; read it with dasc_refresh_status after
- *   synchronising the stream.
+ *   out, or a log-decay outside the chunked kernel's range, sets a flag in
+ *   the workspace; read it with dasc_refresh_status after synchronising the
+ *   stream.
  */
 dasc_status_t dasc_refresh_workspace_bytes(const dasc_plan_t *plan, int32_t n_req, int32_t n_layers_in_call,
                                            int32_t algo, size_t *out);
@@ -326,9 +331,10 @@ dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t l
                            int32_t max_seqlen, int32_t layer_begin, int32_t layer_end, float q_scale,
                            void *o, int32_t o_dtype, int32_t mode, int32_t algo, void *workspace,
                            size_t workspace_bytes, void *cuda_stream);
-/* After the stream has been synchronised: DASC_OK, or DASC_ERR_TIMEOUT if a
- * device-side wait of the last dasc_refresh that used `workspace` gave up.
- * Copies 4 bytes device -> host (synchronous). */
+/* After the stream has been synchronised: DASC_OK; DASC_ERR_TIMEOUT if a
+ * device-side wait of the last dasc_refresh that used `workspace` gave up;
+ * else DASC_ERR_DOMAIN if that call met a log-decay outside the chunked
+ * kernel's range.  Copies 8 bytes device -> host (synchronous). */
 dasc_status_t dasc_refresh_status(const void *workspace, size_t workspace_bytes);
 
 /*

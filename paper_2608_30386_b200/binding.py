@@ -23,7 +23,7 @@ IO_BF16, IO_FP32 = 0, 1
 REFRESH_CONTINUE, REFRESH_SCRATCH_MERGE_LOCAL = 0, 1
 ALGO_AUTO, ALGO_SEQUENTIAL, ALGO_CHUNKED = 0, 1, 2
 
-OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT = range(8)
+OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT, ERR_DOMAIN = range(9)
 
 # Every symbol include/dasc.h declares.
 EXPORTS = (

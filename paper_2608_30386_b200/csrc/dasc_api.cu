@@ -430,9 +430,10 @@ dasc_status_t dasc_refresh_window(const dasc_plan_t *plan, float *state_base, in
 
 dasc_status_t dasc_refresh_status(const void *workspace, size_t workspace_bytes) {
   if (!workspace || workspace_bytes < 4) return DASC_OK;  // nothing was recorded
-  uint32_t flag = 0;
-  if (cudaMemcpy(&flag, workspace, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return DASC_ERR_CUDA;
-  return flag == 0 ? DASC_OK : DASC_ERR_TIMEOUT;
+  uint32_t flag[2] = {0, 0};  // [0] a wait timed out, [1] log-decay out of range
+  if (cudaMemcpy(flag, workspace, workspace_bytes < 8 ? 4 : 8, cudaMemcpyDeviceToHost) != cudaSuccess) return DASC_ERR_CUDA;
+  if (flag[0] != 0) return DASC_ERR_TIMEOUT;
+  return flag[1] == 0 ? DASC_OK : DASC_ERR_DOMAIN;
 }
 
 const char *dasc_status_string(dasc_status_t s) {
@@ -445,6 +446,7 @@ const char *dasc_status_string(dasc_status_t s) {
     case DASC_ERR_CUDA: return "CUDA error";
     case DASC_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case DASC_ERR_TIMEOUT: return "device-side wait timed out";
+    case DASC_ERR_DOMAIN: return "log-decay outside the chunked kernel's range";
   }
   return "unknown status";
 }

@@ -70,6 +70,10 @@ constexpr uint32_t kMaxPolls = 1u << 22;
 // significand, log-uniform in [1, 2)).  The rows of Kt and Qt, the only partners of that operand,
 // are scaled up by this factor to cancel the bias; A and P, which also come from those rows, are
 // scaled back down when they are taken out of TMEM.
+// Largest |sum of the log-decay over half a chunk| per channel for which every factor formed relative to the chunk
+// midpoint stays a normal fp32 number with room for the products that follow.
+constexpr float kMaxHalfDecay = 80.f;
+
 constexpr float kTruncComp = 1.000352f;
 constexpr float kInvTruncComp = 1.0f / kTruncComp;
 constexpr float kLog2TruncComp = 5.0774e-4f;  // log2(kTruncComp)
@@ -481,6 +485,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       PT(2);
       // sums: this lane's total, the prefix over the four token groups of the warp (lanes 8 apart), the half's total
       float run0[2][4], refL[4];
+      bool out_of_range = false;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         float own[4] = {0.f, 0.f, 0.f, 0.f};
@@ -506,6 +511,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           run0[half][i] = incl - own[i];                      // accumulated before this lane's first token
           tot[i] = __shfl_sync(0xffffffffu, incl, cq + 24);    // the half's total
           if (half == 0) refL[i] = -tot[i] * LOG2E;            // minus the midpoint reference, in log2 units
+          out_of_range |= !(fabsf(tot[i]) <= kMaxHalfDecay);   // also true for NaN
         }
         if (half == 0) {
           // The factor that takes the state from where the previous chunk left it to this chunk's midpoint needs
@@ -585,6 +591,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
               make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
       }
       PT(4);
+      if (out_of_range && tg == 0 && err) atomicExch(err + 1, 1u);  // the exponents of this chunk may have overflowed
       fence_smem_to_async();
       mbar_arrive(&misc->rdy_prep);  // -> MMA1
       PT(5);
@@ -812,7 +819,7 @@ int launch(const DascRefreshArgs &a, void *stream) {
   const int64_t n_units = static_cast<int64_t>(a.n_req) * a.n_layers_in_call * a.H_v;
   if (n_units == 0) return cudaSuccess;
   if (n_units > 2147483647LL) return static_cast<int>(cudaErrorInvalidConfiguration);
-  e = cudaMemsetAsync(a.workspace, 0, 4, static_cast<cudaStream_t>(stream));  // clear the time-out flag
+  e = cudaMemsetAsync(a.workspace, 0, 8, static_cast<cudaStream_t>(stream));  // clear the time-out and range flags
   if (e != cudaSuccess) return static_cast<int>(e);
   kern<<<static_cast<unsigned>(n_units), NT, SMEM_ALLOC, static_cast<cudaStream_t>(stream)>>>(a);
   return static_cast<int>(cudaGetLastError());
@@ -820,7 +827,8 @@ int launch(const DascRefreshArgs &a, void *stream) {
 
 }  // namespace
 
-// Scratch the chunked kernel needs: one 32-bit time-out flag (first word), padded to 256 bytes.
+// Scratch the chunked kernel needs: a 32-bit time-out flag (first word) and a 32-bit out-of-range flag (second
+// word), padded to 256 bytes.
 size_t dasc_refresh_chunked_workspace_bytes(int32_t, int32_t, int32_t) { return 256; }
 
 // Returns a cudaError_t as int, or -1 if this kernel does not take the request

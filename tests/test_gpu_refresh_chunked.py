@@ -78,3 +78,31 @@ def test_chunked_matches_sequential_and_auto_picks_it():
             ref = ref_o[0, t0:t1, h]
             bound = TOL * np.abs(ref).max() + np.abs(ref) * 2.0 ** -8
             assert np.all(np.abs(got_o[0, t0:t1, h] - ref) <= bound)
+
+
+def test_log_decay_outside_the_chunked_range_is_reported():
+    # one channel of one head decays by e^-7 per token: 112 over half a chunk, beyond the 80 the midpoint
+    # reference can hold in fp32.  The call must say so (DASC_ERR_DOMAIN from the status query); the same streams
+    # go through the sequential kernel without complaint and match the oracle.
+    import paper_2608_30386_b200.binding as binding
+    case = make_refresh_case(31, dasc.KDA, 1, 2, 2, 128, 128, [64], scope=dasc.SCOPE_LAYER, keep_ratio=0.5)
+    case.streams.g[0, :, 1, 5] = -7.0
+    dev = case.state0.device
+    s = case.streams
+    state = case.state0.clone()
+    ws = torch.zeros(256, dtype=torch.uint8, device=dev)
+    dasc.dasc_refresh(case.plan, state, 2 * 128 * 128, 2 * 128 * 128, torch.arange(1, dtype=torch.int32, device=dev),
+                      s.q, s.k, s.v, s.g, s.beta, case.cu.to(dev), 64, 64, o=None, algo=dasc.ALGO_CHUNKED, workspace=ws)
+    torch.cuda.synchronize()
+    assert dasc.dasc_refresh_status(ws) == binding.ERR_DOMAIN
+    assert dasc.status_string(binding.ERR_DOMAIN) == "log-decay outside the chunked kernel's range"
+    # a call inside the range clears the flag again
+    case.streams.g[0, :, 1, 5] = -1.0
+    dasc.dasc_refresh(case.plan, state, 2 * 128 * 128, 2 * 128 * 128, torch.arange(1, dtype=torch.int32, device=dev),
+                      s.q, s.k, s.v, s.g, s.beta, case.cu.to(dev), 64, 64, o=None, algo=dasc.ALGO_CHUNKED, workspace=ws)
+    torch.cuda.synchronize()
+    assert dasc.dasc_refresh_status(ws) == binding.OK
+    case.streams.g[0, :, 1, 5] = -7.0
+    ref_s, ref_o = run_refresh_oracle(case)
+    got_s, got_o = run_refresh_gpu(case, algo=dasc.ALGO_SEQUENTIAL)
+    assert_refresh_close(case, got_s, got_o, ref_s, ref_o, TOL)
