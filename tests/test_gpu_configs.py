@@ -201,6 +201,14 @@ def test_kda_serving_config_refresh_in_the_benchmarks_launch():
     worst_o = check_sampled_refresh(dasc.KDA, plan, oplan, before, active, ls, rs, q, k, v, g, beta, o, cu, units,
                                     TOL + 2.0 ** -8)
     print(f"KDA serving config, one launch: worst sampled state err {worst:.2e}, with bf16 outputs {worst_o:.2e}")
+    # the same launch once more: every one of the 49,152 states and all outputs must come out with the same bits
+    again, o2 = before.clone(), torch.empty_like(o)
+    dasc.dasc_refresh(plan, again, ls, rs, ids, q, k, v, g, beta, cu.to(dev), T, suffix, o=o2, workspace=ws)
+    torch.cuda.synchronize()
+    assert dasc.dasc_refresh_status(ws) == 0
+    assert torch.equal(again.view(torch.int32), active.view(torch.int32))
+    assert torch.equal(o2.view(torch.int16), o.view(torch.int16))
+    del again, o2
     # the paper's load policy on the same launch shape: scratch replay of the same 256 tokens, no outputs
     merged = before.clone()
     wb = torch.empty(n_req, dtype=torch.int32, device=dev)
