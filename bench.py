@@ -47,8 +47,8 @@ CHUNKED_FLOPS_PER_TOKEN_HEAD = 196608   # tf32 flops the chunked kernel issues p
 # the KDA serving workload at 8 requests and a 128-token suffix (a full-size launch is too large to capture); every
 # request and token moves the same bytes, so traffic grows in proportion and a full launch is scaled by its units.
 # Below 1.0 = lines still dirty in L2 when the kernel ended, not skipped work.
-NCU_TRAFFIC_OVER_ALGORITHMIC = {"pack": 254.99e6 / 306.12e6, "restore": 499.80e6 / 555.71e6,
-                                "refresh_chunked": 1.9815e9 / 2.0164e9}
+NCU_TRAFFIC_OVER_ALGORITHMIC = {"pack": 255.99e6 / 306.12e6, "restore": 500.13e6 / 555.71e6,
+                                "refresh_chunked": 1.9830e9 / 2.0164e9}
 
 CONFIGS = {
     1: dict(name="kda_serving", kind="KDA", L=24, H_v=32, H_k=32, n_req=64, keep=0.38, rate_lo=1e-3, suffix=256, seed=1),
