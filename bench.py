@@ -448,33 +448,50 @@ def main():
         n_e = min(16, N_REQ)                                 # requests per e2e step (bounded pinned memory)
         Te = n_e * SUFFIX
         ge = min(group, 6)                                   # layers of token streams copied per refresh call
-        h_state = torch.empty((L, n_e, dense), dtype=torch.float32).pin_memory()
-        h_state.copy_(state[:, :n_e])
+        # request-major on both sides, so that a group of requests is one contiguous transfer
+        h_state = torch.empty((n_e, L, dense), dtype=torch.float32).pin_memory()
+        h_state.copy_(state[:, :n_e].transpose(0, 1))
         host_streams = [x[:ge, :Te].contiguous().cpu().pin_memory() for x in (q, k, v, g, beta)]
         pool_shape, pool_dtype = ((n_e, slot_bytes), torch.uint8) if int8 else ((n_e, slot), torch.float32)
         h_pool = torch.empty(pool_shape, dtype=pool_dtype).pin_memory()
-        h_out = torch.empty((L, n_e, dense), dtype=torch.float32).pin_memory()
+        h_out = torch.empty((n_e, L, dense), dtype=torch.float32).pin_memory()
         h_o = torch.empty((ge, Te, H_v, D), dtype=torch.bfloat16).pin_memory()
-        d_state = torch.empty((L, n_e, dense), device=dev)
+        d_state = torch.empty((n_e, L, dense), device=dev)
         d_active = torch.empty_like(d_state)
         d_pool = torch.empty(pool_shape, dtype=pool_dtype, device=dev)
         d_streams = [torch.empty(x.shape, dtype=x.dtype, device=dev) for x in host_streams]
         d_o = torch.empty((ge, Te, H_v, D), dtype=torch.bfloat16, device=dev)
         cu_e = synth.uniform_cu_seqlens(n_e, SUFFIX).to(dev)
         ids_e = torch.arange(n_e, dtype=torch.int32, device=dev)
-        ls_e = n_e * dense
+        ls_e, rs_e = dense, L * dense
+        # Store / Load in `parts` groups of requests: group i's pool goes back to the host on a second stream while
+        # group i+1's states are still coming in (PCIe carries both directions at once)
+        parts = 4 if (args.layout == "ragged" and n_e % 4 == 0) else 1
+        s_out = torch.cuda.Stream(device=dev)
+        part_done = [torch.cuda.Event() for _ in range(parts)]
+        out_done = torch.cuda.Event()
+        part_ids = [ids_e[i * (n_e // parts):(i + 1) * (n_e // parts)].contiguous() for i in range(parts)]
 
         def e2e_step(ev):
             ev[0].record(stream)
-            d_state.copy_(h_state, non_blocking=True)
-            do_pack(plan, d_state, ls_e, dense, ids_e, d_pool, ids_e)
-            do_restore(plan, d_pool, ids_e, d_active, ls_e, dense, ids_e)
-            h_pool.copy_(d_pool, non_blocking=True)
+            s_out.wait_stream(stream)                          # the previous step has let go of the pool buffers
+            for i in range(parts):
+                a0, a1 = i * (n_e // parts), (i + 1) * (n_e // parts)
+                d_state[a0:a1].copy_(h_state[a0:a1], non_blocking=True)
+                do_pack(plan, d_state, ls_e, rs_e, part_ids[i], d_pool, part_ids[i])
+                do_restore(plan, d_pool, part_ids[i], d_active, ls_e, rs_e, part_ids[i])
+                part_done[i].record(stream)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(part_done[i])
+                    h_pool[a0:a1].copy_(d_pool[a0:a1], non_blocking=True)
+            with torch.cuda.stream(s_out):
+                out_done.record(s_out)
+            stream.wait_event(out_done)
             ev[1].record(stream)
             for gi in range(L // ge):                        # every layer group: its streams in, its outputs out
                 for dst, src in zip(d_streams, host_streams):
                     dst.copy_(src, non_blocking=True)
-                dasc.dasc_refresh(plan, d_active, ls_e, dense, ids_e, *d_streams, cu_e, Te, SUFFIX,
+                dasc.dasc_refresh(plan, d_active, ls_e, rs_e, ids_e, *d_streams, cu_e, Te, SUFFIX,
                                   layer_begin=gi * ge, layer_end=(gi + 1) * ge, o=d_o, algo=algo, workspace=ws)
                 h_o.copy_(d_o, non_blocking=True)
             h_out.copy_(d_active, non_blocking=True)
@@ -496,7 +513,8 @@ def main():
         e2e = {"value": world * e_bytes / (t_copy * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "requests_per_step": n_e,
                "refresh_tokens_per_s": world * Te / (t_ref * 1e-3), "ms_pack_restore": t_copy, "ms_refresh": t_ref,
-               "note": "pinned host buffers; H2D of states and token streams, D2H of pool, states and outputs timed"}
+               "note": "pinned host buffers; H2D of states and token streams, D2H of pool, states and outputs timed; "
+                       "Store/Load in request groups, a group's pool read back while the next group uploads"}
         del h_state, host_streams, h_pool, h_out, h_o, d_state, d_active, d_pool, d_streams, d_o
 
     if rank != 0:
