@@ -46,6 +46,8 @@ def lib():
         _lib.oracle_replay_window_unit.argtypes = [C.c_double, C.c_double]
         _lib.oracle_slot_budget.restype = C.c_int64
         _lib.oracle_max_threads.restype = C.c_int32
+        _lib.oracle_splitmix64.restype = C.c_uint64
+        _lib.oracle_splitmix64.argtypes = [C.c_uint64]
     return _lib
 
 
@@ -62,6 +64,11 @@ def horizon(A_log, dt_bias, a=-0.3, eps=1e-3):
     lib().oracle_horizon(C.c_int64(A_log.size), _p(A_log), _p(dt_bias), C.c_double(a),
                          C.c_double(eps), _p(g), _p(Hs))
     return g, Hs
+
+
+def splitmix64(x: int) -> int:
+    """The key function of the count-matched random selector (Appendix C.3 control)."""
+    return int(lib().oracle_splitmix64(C.c_uint64(x & 0xFFFFFFFFFFFFFFFF)))
 
 
 def replay_window_unit(Hs: float, w_max: float) -> float:

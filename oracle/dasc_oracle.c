@@ -98,6 +98,11 @@ static uint64_t splitmix64(uint64_t x)
     return x ^ (x >> 31);
 }
 
+/* The same function, exported so that a test can hold it against the generator's
+ * published outputs (the n-th output of a generator seeded s is splitmix64 of
+ * s + (n-1) * 0x9E3779B97F4A7C15). */
+uint64_t oracle_splitmix64(uint64_t x) { return splitmix64(x); }
+
 /* Keep the r units of a group with the largest score; ties go to the lower
  * index.  Deliberately O(n^2): rank by counting, no sort to get wrong. */
 static void keep_top(const double *score, int64_t n, int64_t r, uint8_t *mask)

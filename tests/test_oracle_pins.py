@@ -103,6 +103,53 @@ def test_replay_window_matches_table8_reading():
     assert p.mask.all() and p.W_replay == 0
 
 
+def _a_log_for_horizons(hs):
+    """A_log (fp32) whose Eq. 3 horizon with a = -0.3, dt_bias = 0 is `hs` (to fp32 rounding): H_s = 12.4609 / rate."""
+    return np.log(12.46088198480878 / np.asarray(hs, np.float64)).astype(np.float32)
+
+
+def test_window_cap_of_a_non_threshold_plan_is_taken_from_the_omitted_units_only():
+    # Eq. 7 needs a cap W_max; a plan that was not built by the threshold rule has none, and the reading taken is
+    # cap = next power of two of the LARGEST OMITTED horizon, floored at 4 (Section 4.2: the window is sized for the
+    # local units that are replayed, and it is at least 4 tokens).  Hand-built horizons, explicit masks.
+    hs = [5.0, 20.0, 100.0, 300.0, 3.0, 1000.0]
+    A = _a_log_for_horizons(hs).reshape(1, 6)
+    Z = np.zeros_like(A)
+    keep = np.array([[0, 0, 0, 1, 0, 1]], np.uint8)            # the two longest horizons are retained
+    p = oracle.plan(oracle.GDN, 1, 6, 1, A, Z, sel=oracle.SEL_EXPLICIT, explicit_mask=keep, w_max=0.0)
+    np.testing.assert_allclose(p.Hs.ravel(), hs, rtol=1e-6)
+    assert p.w_max_used == 128                                  # next_pow2(100); NOT 1024 = next_pow2 of a retained unit
+    assert p.W_replay == 128
+    np.testing.assert_array_equal(p.W_u.ravel(), [8, 32, 128, 128, 4, 128])   # retained units are clamped to the cap too
+    # retaining the 100-token unit as well lowers the cap to next_pow2(20) = 32
+    keep2 = np.array([[0, 0, 1, 1, 0, 1]], np.uint8)
+    p = oracle.plan(oracle.GDN, 1, 6, 1, A, Z, sel=oracle.SEL_EXPLICIT, explicit_mask=keep2, w_max=0.0)
+    assert p.w_max_used == 32 and p.W_replay == 32
+    np.testing.assert_array_equal(p.W_u.ravel(), [8, 32, 32, 32, 4, 32])
+    # only very short horizons omitted: next_pow2(3) = 4; next_pow2(1.5) = 2 is floored at 4
+    for omitted_h, in ((3.0,), (1.5,)):
+        A2 = _a_log_for_horizons([omitted_h, 50.0, 70.0]).reshape(1, 3)
+        p = oracle.plan(oracle.GDN, 1, 3, 1, A2, np.zeros_like(A2), sel=oracle.SEL_EXPLICIT,
+                        explicit_mask=np.array([[0, 1, 1]], np.uint8), w_max=0.0)
+        assert p.w_max_used == 4 and p.W_replay == 4
+    # nothing omitted: nothing to replay
+    p = oracle.plan(oracle.GDN, 1, 6, 1, A, Z, sel=oracle.SEL_EXPLICIT, explicit_mask=np.ones((1, 6), np.uint8), w_max=0.0)
+    assert p.W_replay == 0
+    # a cap given by the caller is used as it is, also with a non-threshold rule
+    p = oracle.plan(oracle.GDN, 1, 6, 1, A, Z, sel=oracle.SEL_EXPLICIT, explicit_mask=keep, w_max=16.0)
+    assert p.w_max_used == 16 and p.W_replay == 16
+    np.testing.assert_array_equal(p.W_u.ravel(), [8, 16, 16, 16, 4, 16])
+    # the same through the top-ratio rule: 8 units in two layers, keep half per layer -> the two shortest of each
+    # layer are omitted; the largest omitted horizon is 40 -> cap 64, although 900 and 600 are present
+    hs8 = [[900.0, 7.0, 40.0, 600.0], [33.0, 2.0, 500.0, 34.0]]
+    A8 = _a_log_for_horizons(hs8)
+    p = oracle.plan(oracle.GDN, 2, 4, 1, A8, np.zeros_like(A8), sel=oracle.SEL_TOP_RATIO, keep_ratio=0.5,
+                    scope=oracle.SCOPE_LAYER, w_max=0.0)
+    np.testing.assert_array_equal(p.mask, [[1, 0, 0, 1], [0, 0, 1, 1]])
+    assert p.w_max_used == 64 and p.W_replay == 64
+    np.testing.assert_array_equal(p.W_u, [[64, 8, 64, 64], [64, 4, 64, 64]])
+
+
 # ----------------------------------------------------------------------------
 # Section 4.1 selection, Appendix B offsets, Eq. 6 ratios
 # ----------------------------------------------------------------------------
@@ -172,6 +219,49 @@ def test_top_ratio_brute_force_and_ties():
                     np.zeros((1, 256), np.float32), sel=oracle.SEL_TOP_RATIO, keep_ratio=0.4,
                     scope=oracle.SCOPE_HEAD)
     np.testing.assert_array_equal(p.mask.reshape(4, 64).sum(1), [26] * 4)
+
+
+@pytest.mark.parametrize("ratio,n,want", [(0.4, 5, 2), (0.38, 4096, 1557), (0.25, 4096, 1024), (0.2, 4096, 820),
+                                          (0.5, 32, 16), (0.4, 64, 26), (0.0, 7, 0), (1.0, 7, 7)])
+def test_top_ratio_count_hand_values(ratio, n, want):
+    # "keep the ceil(ratio * n) longest horizons", where a product that is an integer up to rounding noise counts as
+    # that integer: 0.4 * 5 = 2.0000000000000004 in binary floating point keeps 2 units, not 3.  The counts below are
+    # computed by hand (0.38 * 4096 = 1556.48, 0.2 * 4096 = 819.2, 0.4 * 64 = 25.6).
+    rng = np.random.default_rng(5)
+    rates = np.exp(rng.uniform(math.log(1e-3), 0.0, size=(1, n))).astype(np.float32)
+    p = oracle.plan(oracle.GDN, 1, n, 1, np.log(rates), np.zeros_like(rates), sel=oracle.SEL_TOP_RATIO,
+                    keep_ratio=ratio, scope=oracle.SCOPE_LAYER)
+    assert p.sum_r == want == p.r_l[0]
+    if 0 < want < n:
+        kept, dropped = p.Hs[p.mask == 1], p.Hs[p.mask == 0]
+        assert kept.min() >= dropped.max()                      # the kept ones are the longest horizons
+
+
+def test_random_selector_key_function_known_answers():
+    # the key function is the published splitmix64 generator: its reference outputs pin the three constants, the
+    # shifts and the order of the steps
+    gamma = 0x9E3779B97F4A7C15
+    with open(os.path.join(os.path.dirname(GOLDEN), "splitmix64_known_answers.txt")) as f:
+        rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    assert len(rows) >= 7
+    for seed, n, value in rows:
+        assert oracle.splitmix64(int(seed) + (int(n) - 1) * gamma) == int(value)
+    # and the plan keys unit u of layer l with splitmix64(seed + (l << 32) + u), smallest keys retained:
+    # two units, one kept, seed 0 -> keys 0xE220A8397B1DCDAF (unit 0) and 0x910A2DEC89025CC1 (unit 1): unit 1 stays
+    A = np.zeros((1, 2), np.float32)
+    p = oracle.plan(oracle.GDN, 1, 2, 1, A, A, sel=oracle.SEL_TOP_RATIO, keep_ratio=0.5, randomize=True, seed=0)
+    np.testing.assert_array_equal(p.mask, [[0, 1]])
+    # a seed chosen so that unit 0's key is the generator's 3rd output for 1234567 (9817491932198370423, above 2^63)
+    # and unit 1 of layer 0 gets ... whatever the pinned function says; the mask must follow the pinned keys
+    for seed in (1234567 + 2 * gamma, 1234567, 42):
+        L, n = 3, 5
+        A = np.zeros((L, n), np.float32)
+        p = oracle.plan(oracle.GDN, L, n, 1, A, A, sel=oracle.SEL_TOP_RATIO, keep_ratio=0.4, randomize=True, seed=seed)
+        for l in range(L):
+            keys = [oracle.splitmix64(seed + (l << 32) + u) for u in range(n)]
+            want = np.zeros(n, np.uint8)
+            want[np.argsort(keys, kind="stable")[:2]] = 1
+            np.testing.assert_array_equal(p.mask[l], want)
 
 
 def test_random_selector_is_count_matched_and_seeded():
