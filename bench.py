@@ -290,7 +290,18 @@ def main():
                     help="imbalanced per-layer decay profile: layer rates scaled by exp(skew * (l/(L-1) - 1/2))")
     ap.add_argument("--codec", default="fp32", choices=["fp32", "int8"],
                     help="checkpoint pool format: fp32 bit copies, or the Appendix D INT8 codec fused into pack/restore")
+    ap.add_argument("--pool-slots", type=int, default=2048, help="config 4: slots of the bounded checkpoint pool")
+    ap.add_argument("--trace-rounds", type=int, default=0, help="config 4: replay only the first rounds of the trace")
+    ap.add_argument("--dry-launch", action="store_true", help="start the ranks, count them over gloo, do no GPU work")
     args = ap.parse_args()
+    world_env = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and world_env == 1 and "DASC_BENCH_SPAWNED" not in os.environ:
+        sys.exit(spawn_replicas(args.gpus))                 # no launcher around us: start the N ranks ourselves
+    if args.gpus != world_env:
+        raise SystemExit(f"--gpus {args.gpus} does not match the {world_env} rank(s) that were launched")
+    if args.dry_launch:
+        dry_launch(args)
+        return
     c = dict(CONFIGS[args.config])
     if args.requests is not None:
         c["n_req"] = args.requests
@@ -368,7 +379,7 @@ def main():
     o = torch.empty((group, T, H_v, D), dtype=torch.bfloat16, device=dev)
     cu = synth.uniform_cu_seqlens(N_REQ, SUFFIX).to(dev)
     ws_bytes = dasc.dasc_refresh_workspace_bytes(plan, N_REQ, group, algo)
-    ws = torch.zeros(max(ws_bytes, 256), dtype=torch.uint8, device=dev) if ws_bytes else None
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev) if ws_bytes else None
 
     pack_bytes = N_REQ * (slot * 4 + slot_bytes)
     restore_bytes = N_REQ * (slot_bytes + L * dense * 4)
@@ -588,7 +599,9 @@ def main():
         "window_refresh_state_only": {"ms": t_window, "tokens_per_s": world * N_REQ * SUFFIX / (t_window * 1e-3),
                                       "token_heads_per_s": world * token_heads / (t_window * 1e-3)},
         "roofline": roofline, "roofline_by_kernel": rl, "clocks": clocks,
-        "gpu_launches": (2 + n_groups) * args.steps,
+        # per step: pack, restore, and per layer group the tensor-core refresh kernel + the exact kernel's pass over
+        # the units handed to it (AUTO); a single refresh kernel per group when an algorithm is forced
+        "gpu_launches": (2 + n_groups * (2 if args.algo == "auto" else 1)) * args.steps,
     }
     if e2e:
         line["e2e"] = e2e
@@ -600,9 +613,16 @@ def main():
 
 
 def run_mixed_trace(args, c):
-    """Mixed serving trace (single GPU): waves of new checkpoints are packed on one stream while cached
-    checkpoints are restored and refreshed (ragged suffixes, uniform in [1, 1024]) on another.  The slot pool is
-    one contiguous buffer recycled round-robin.  Reports both streams overlapped and run one after the other."""
+    """Mixed serving trace (single GPU; Appendix C.1: a bounded pool of checkpoint slots with LRU recycling).
+
+    The event list comes from `synth.serving_trace` (seed 4): 512 requests with prefix lengths log-uniform in
+    [1 Ki, 128 Ki], one checkpoint stored every 1024 tokens, follow-up requests that hit the newest resident
+    checkpoint of a shared prefix and replay the 1..1024 tokens since it.  The list is cut into rounds whose two
+    sides are independent: new checkpoints are packed on one stream (the higher-priority one) while hits are restored
+    and refreshed (ragged suffixes) on another.  A step is one replay of the whole trace; it is timed with the
+    two streams overlapped and with each round's two sides run one after the other.  Checkpoint contents and token
+    values do not affect the time: the states of a round's new checkpoints and the token streams are fixed synthetic
+    buffers (six layers of streams resident, reused by every layer group and round)."""
     import paper_2608_30386_b200 as dasc
     from paper_2608_30386_b200 import synth
 
@@ -611,84 +631,170 @@ def run_mixed_trace(args, c):
         return
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    pk = peaks()
-    L, H, wave, n_slots = c["L"], c["H_v"], c["n_req"], 1024
+    L, H, batch = c["L"], c["H_v"], c["n_req"]
+    n_slots = args.pool_slots
     plan, rates, gen = build_plan(c, local)
+    rounds, tstats = synth.serving_trace(c["seed"], n_slots=n_slots, batch=batch)
+    if args.trace_rounds:
+        rounds = rounds[:args.trace_rounds]
     dense = H * D * D
-    ls, rs = wave * dense, dense
+    ls, rs = batch * dense, dense
     slot = int(plan.slot_floats)
     dgen = synth.generator(c["seed"], dev)
     pool = torch.empty((n_slots, slot), device=dev)
-    pool.normal_(generator=dgen)                                       # resident checkpoints to hit
-    new_states = synth.states(dgen, (L, wave, dense), dev)
-    active = torch.empty((L, wave, dense), device=dev)
-    ids = torch.arange(wave, dtype=torch.int32, device=dev)
-    n_waves = args.warmup + args.steps
-    cus = [synth.ragged_cu_seqlens(gen, wave, 1, 1024) for _ in range(n_waves)]
-    t_max = max(int(cu[-1]) for cu in cus)
+    pool.normal_(generator=dgen)
+    new_states = synth.states(dgen, (L, batch, dense), dev)
+    active = torch.empty((L, batch, dense), device=dev)
+    ids = torch.arange(batch, dtype=torch.int32, device=dev)
+    t_max = max(max(sum(r.suffix) for r in rounds), 1)
     group = 6                                                          # layers of token streams resident at once
     parts = [synth.token_streams(dgen, synth.KDA, 1, t_max, H, H, D, D, rates[l:l + 1], device=dev) for l in range(group)]
     q, k, v, g, beta = (torch.cat([getattr(p, f) for p in parts]) for f in ("q", "k", "v", "g", "beta"))
     del parts
     o = torch.empty((group, t_max, H, D), dtype=torch.bfloat16, device=dev)
-    ws = torch.zeros(256, dtype=torch.uint8, device=dev)
-    s_pack, s_load = torch.cuda.Stream(), torch.cuda.Stream()
-    cu_dev = [cu.to(dev) for cu in cus]
-    new_slots = [((torch.arange(wave) + 512 + w * wave) % 512 + 512).to(torch.int32).to(dev) for w in range(n_waves)]
-    hit_slots = [torch.randperm(512, generator=gen)[:wave].to(torch.int32).to(dev) for _ in range(n_waves)]
+    ws = torch.zeros(dasc.dasc_refresh_workspace_bytes(plan, batch, group), dtype=torch.uint8, device=dev)
+    # the copy stream gets the higher priority: its blocks are placed as soon as a refresh CTA retires
+    lo_pri, hi_pri = torch.cuda.Stream.priority_range() if hasattr(torch.cuda.Stream, "priority_range") else (0, -1)
+    s_pack = torch.cuda.Stream(priority=hi_pri)
+    s_load = torch.cuda.Stream(priority=lo_pri)
+    dev_rounds = []
+    for r in rounds:
+        cu = torch.zeros(len(r.suffix) + 1, dtype=torch.int64)
+        cu[1:] = torch.cumsum(torch.tensor(r.suffix, dtype=torch.int64), 0) if r.suffix else cu[1:]
+        dev_rounds.append((torch.tensor(r.store_slots, dtype=torch.int32, device=dev),
+                           torch.tensor(r.hit_slots, dtype=torch.int32, device=dev), cu.to(torch.int32).to(dev),
+                           max(r.suffix) if r.suffix else 0))
+    launches = 0
 
-    def pack_side(w):
-        dasc.dasc_pack(plan, new_states, ls, rs, ids, pool, new_slots[w], stream=s_pack)
+    def store_side(i):
+        nonlocal launches
+        slots = dev_rounds[i][0]
+        n = int(slots.numel())
+        if n:
+            dasc.dasc_pack(plan, new_states, ls, rs, ids[:n], pool, slots, stream=s_pack)
+            launches += 1
 
-    def load_side(w):
-        T = int(cus[w][-1])
-        # streams are laid out for t_max tokens per layer; the call sees the first T of each layer
-        dasc.dasc_restore(plan, pool, hit_slots[w], active, ls, rs, ids, stream=s_load)
-        for gi in range(L // group):
-            dasc.dasc_refresh(plan, active, ls, rs, ids, q, k, v, g, beta, cu_dev[w], t_max, 1024,
+    def load_side(i):
+        nonlocal launches
+        _, hits, cu, longest = dev_rounds[i]
+        n = int(hits.numel())
+        if not n:
+            return
+        dasc.dasc_restore(plan, pool, hits, active, ls, rs, ids[:n], stream=s_load)
+        launches += 1
+        for gi in range(L // group):       # the streams hold t_max tokens per layer; the call sees this round's first T
+            dasc.dasc_refresh(plan, active, ls, rs, ids[:n], q, k, v, g, beta, cu, t_max, longest,
                               layer_begin=gi * group, layer_end=(gi + 1) * group, o=o, workspace=ws, stream=s_load)
+            launches += 2
 
-    def run(overlap):
+    def replay(overlap):
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        for w in range(args.warmup):
-            pack_side(w)
-            load_side(w)
         torch.cuda.synchronize()
-        ev0.record(torch.cuda.current_stream())
+        main = torch.cuda.current_stream()
+        ev0.record(main)
         s_pack.wait_event(ev0)
         s_load.wait_event(ev0)
-        for w in range(args.warmup, n_waves):
-            pack_side(w)
+        for i in range(len(rounds)):
+            store_side(i)
             if not overlap:
                 s_load.wait_stream(s_pack)
-            load_side(w)
-            if not overlap:
-                s_pack.wait_stream(s_load)
-        torch.cuda.current_stream().wait_stream(s_pack)
-        torch.cuda.current_stream().wait_stream(s_load)
-        ev1.record(torch.cuda.current_stream())
+            load_side(i)
+            # a round's two sides are independent of each other, consecutive rounds are not
+            s_pack.wait_stream(s_load)
+            s_load.wait_stream(s_pack)
+        main.wait_stream(s_pack)
+        main.wait_stream(s_load)
+        ev1.record(main)
         torch.cuda.synchronize()
-        return ev0.elapsed_time(ev1) / args.steps
+        return ev0.elapsed_time(ev1)
 
+    steps = max(1, min(args.steps, 3))
+    replay(True)                                                       # warm-up: one whole trace
     sampler = ClockSampler(local)
     sampler.start()
-    t_serial = run(False)
-    t_overlap = run(True)
+    launches = 0
+    t_overlap = sum(replay(True) for _ in range(steps)) / steps
+    counted = launches // steps
+    t_serial = sum(replay(False) for _ in range(steps)) / steps
+    # each side alone, for the overlap bound: max(copy, load) <= overlapped <= copy + load
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    torch.cuda.synchronize()
+    ev[0].record(s_pack)
+    for i in range(len(rounds)):
+        store_side(i)
+    ev[1].record(s_pack)
+    s_load.wait_event(ev[1])
+    for i in range(len(rounds)):
+        load_side(i)
+    ev[2].record(s_load)
+    torch.cuda.synchronize()
+    t_store, t_load = ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2])
     clocks = sampler.stop()
     assert dasc.dasc_refresh_status(ws) == 0
-    tokens = sum(int(cu[-1]) for cu in cus[args.warmup:]) / args.steps
-    copy_bytes = (2 * wave * slot + wave * (slot + L * dense)) * 4
+    n_store = sum(len(r.store_slots) for r in rounds)
+    n_hit = sum(len(r.hit_slots) for r in rounds)
+    tokens = sum(sum(r.suffix) for r in rounds)
+    copy_bytes = (2 * n_store * slot + n_hit * (slot + L * dense)) * 4
     print(json.dumps({
         "metric": "pack_restore_GBps", "value": copy_bytes / (t_overlap * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": 1,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_overlap, "higher_is_better": True, "scaling": "weak",
+        "steps": steps, "warmup": 1, "ms_per_step": t_overlap, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": workload_name(c), "wave_requests": wave, "pool_slots": n_slots,
-                   "suffix_tokens": "uniform in [1, 1024]", "streams": 2,
-                   "note": "value counts pack+restore bytes over the whole overlapped step, refresh included"},
+        "config": {"workload": workload_name(c), "trace": {k2: v2 for k2, v2 in tstats.items()},
+                   "rounds_replayed": len(rounds), "requests": 512, "prefix_tokens": "log-uniform in [1024, 131072]",
+                   "checkpoint_interval_tokens": 1024, "pool_slots": n_slots, "pool_bytes": pool.numel() * 4,
+                   "recycling": "least recently used (host side)", "round_batch": batch,
+                   "suffix_tokens": "uniform in [1, 1024]", "streams": 2, "copy_stream_priority": hi_pri,
+                   "note": "a step replays the whole trace; value counts pack+restore bytes over the overlapped step, "
+                           "refresh included"},
         "ms_per_step_serial": t_serial, "overlap_speedup": t_serial / t_overlap,
+        "ms_store_side_alone": t_store, "ms_load_side_alone": t_load,
+        "checkpoints_stored": n_store, "hits_served": n_hit,
         "refresh_tokens_per_s": tokens / (t_overlap * 1e-3), "tokens_per_step": tokens, "clocks": clocks,
-        "gpu_launches": (2 + L // group) * args.steps * 2,
+        "gpu_launches": counted * steps,
     }))
+
+
+# ----------------------------------------------------------------------------------------------
+# N > 1 without a launcher: this script starts its own ranks
+# ----------------------------------------------------------------------------------------------
+
+def spawn_replicas(n: int) -> int:
+    """`python bench.py --gpus N` started by hand: run N ranks of this script (one process per GPU, rendezvous on
+    127.0.0.1) and pass rank 0's JSON line through.  Returns the exit code (non-zero if any rank failed)."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port), DASC_BENCH_SPAWNED="1")
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    codes = [p.wait() for p in procs]
+    bad = [(r, code) for r, code in enumerate(codes) if code != 0]
+    if bad:
+        sys.stderr.write(f"bench.py: {len(bad)} of {n} ranks failed (rank, exit code): {bad}\n")
+        return 1
+    return 0
+
+
+def dry_launch(args):
+    """Launcher check that needs no GPU: every rank joins a gloo group and is counted."""
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    count = torch.ones(1, dtype=torch.int64)
+    if world > 1:
+        dist.all_reduce(count)
+    if int(count.item()) != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but {int(count.item())} ranks ran")
+    if rank == 0:
+        print(json.dumps({"dry_launch": True, "n_gpus": args.gpus, "ranks": int(count.item())}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -21,6 +21,9 @@
  *     plan (a plan is immutable after creation).
  *   - Argument errors are detected on the host before any launch and leave
  *     the outputs untouched.
+ *   - Device calls must be made with the plan's device current (cudaSetDevice);
+ *     any other current device is refused with DASC_ERR_INVALID_ARG, because the
+ *     plan's index tables live on that device.
  *   - State orientation: the paper writes the recurrent state as S in
  *     R^{d_v x d_k} with o = S q (Section 3.1).  This library stores the
  *     transpose, S[head][d_k][d_v], fp32, row-major, so that one KDA key
@@ -238,11 +241,78 @@ dasc_status_t dasc_slot_budget(int64_t budget_bytes, const int64_t *temporal_byt
  *                   units each rank stores, consecutive runs in rank order (the split
  *                   sizes of the variable-split all-to-all at Store; its transpose
  *                   is the Load transfer).  The diagonal entry stays on its rank.
- * The exchange itself is not part of this library's device path (one GPU, no
- * collective); the Python package carries a torch.distributed form of it.
+ * dasc_pack_tp / dasc_restore_tp below move the units; the Python package also
+ * carries a torch.distributed (library all-to-all) form of the same transfer.
  */
 dasc_status_t dasc_tp_balance(const int64_t *units_per_rank, int32_t n_ranks, int64_t *slot_width,
                               int64_t *send_counts);
+
+/*
+ * TP-balanced placement, second stage, on the device (Section 4.3: at Store only
+ * remotely owned units cross to another rank; Load applies the inverse transfer
+ * before the compute-local layout is restored).  Rank `rank` of a TP group of
+ * n_ranks packs its retained units as dasc_pack does, but the unit at global
+ * position p = (sum of units_per_rank below `rank`) + (its index in this rank's
+ * packed order) is stored in the pool of rank p / C at local unit index p % C,
+ * C = ceil(sum_r U_r / T): the store goes straight into the owner's pool with
+ * plain 16-byte stores (a push; for another GPU's pool the pointer is a peer
+ * mapping, and nothing but this kernel's stores touches it).  dasc_restore_tp
+ * is the inverse gather with the zero-fill of dasc_restore fused in.
+ *   pool_bases      HOST array of n_ranks DEVICE pointers, 16-byte aligned: base
+ *                   of every rank's pool as seen from this GPU.  n_ranks <= 16.
+ *   units_per_rank  HOST int64[n_ranks]: U_r; entry `rank` must equal this plan's
+ *                   units_retained (every rank has its own plan: its own heads).
+ *   slot_stride     floats between a rank's slots, multiple of 4, >= C*unit_floats;
+ *                   0 = C*unit_floats.  Slot s of a rank holds local units [0, C).
+ * Ordering between ranks is the caller's: a Store is visible to the other ranks'
+ * Loads once its stream has been synchronised and the ranks have met (a barrier
+ * of the caller's process group).  All else as for dasc_pack / dasc_restore.
+ */
+dasc_status_t dasc_pack_tp(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride,
+                           int64_t req_stride, const int32_t *src_req, float *const *pool_bases,
+                           const int64_t *units_per_rank, int32_t n_ranks, int32_t rank,
+                           int64_t slot_stride, const int32_t *dst_slot, int32_t n_pairs,
+                           void *cuda_stream);
+dasc_status_t dasc_restore_tp(const dasc_plan_t *plan, float *const *pool_bases,
+                              const int64_t *units_per_rank, int32_t n_ranks, int32_t rank,
+                              int64_t slot_stride, const int32_t *src_slot, float *state_base,
+                              int64_t layer_stride, int64_t req_stride, const int32_t *dst_req,
+                              int32_t n_pairs, void *cuda_stream);
+
+/*
+ * TP-balanced placement, first stage (Section 4.3: a model-load-time permutation
+ * redistributes linear-attention head bundles across TP ranks, an exact
+ * re-indexing).  The paper does not state how the permutation is chosen; this
+ * library's reading: every rank keeps the same number of bundles per layer (so
+ * compute stays balanced), and bundles are placed greedily, layers in ascending
+ * order, within a layer the bundle with the most retained units first (ties: the
+ * lower index), each on the rank with the smallest payload so far that still
+ * has room in this layer (ties: the lower rank).  Host arithmetic only.
+ *   heads_per_bundle  value heads that must move together (1 for KDA; H_v/H_k
+ *                     for GDN, where a key head and its value heads are coupled);
+ *                     n_v_heads / heads_per_bundle must be a multiple of n_ranks.
+ *   perm              HOST out int32[n_layers][n_bundles]: perm[l][i] = original
+ *                     bundle at position i of layer l; rank r owns positions
+ *                     [r*n_bundles/T, (r+1)*n_bundles/T), ascending original index.
+ *   units_per_rank    HOST out int64[n_ranks]: U_r under this placement.
+ */
+dasc_status_t dasc_tp_head_permutation(const dasc_plan_t *plan, int32_t n_ranks, int32_t heads_per_bundle,
+                                       int32_t *perm, int64_t *units_per_rank);
+
+/*
+ * The convolution state of a checkpoint (Section 4.1: stored uncompressed, in
+ * bf16, beside the temporal state; B_conv of Eq. 6).  To this library it is an
+ * opaque blob of conv_bytes per request:
+ *     pool[dst_slot[i]] = conv[src_req[i]]   (store)      conv[dst_req[i]] = pool[src_slot[i]]   (load)
+ * as bit copies.  Bases DEVICE and 16-byte aligned; conv_bytes and both strides
+ * (bytes between requests / between slots, >= conv_bytes) multiples of 16.
+ */
+dasc_status_t dasc_conv_store(const void *conv_base, int64_t req_stride_bytes, const int32_t *src_req,
+                              void *pool_base, int64_t slot_stride_bytes, const int32_t *dst_slot,
+                              int64_t conv_bytes, int32_t n_pairs, void *cuda_stream);
+dasc_status_t dasc_conv_load(const void *pool_base, int64_t slot_stride_bytes, const int32_t *src_slot,
+                             void *conv_base, int64_t req_stride_bytes, const int32_t *dst_req,
+                             int64_t conv_bytes, int32_t n_pairs, void *cuda_stream);
 
 /*
  * INT8 checkpoint codec fused into the Store / Load copies (Appendix D, Eq. 10).
@@ -304,23 +374,32 @@ dasc_status_t dasc_restore_int8(const dasc_plan_t *plan, const void *pool_base,
  *
  * algo SEQUENTIAL is exact fp32 arithmetic token by token and accepts any g <= 0.
  * algo CHUNKED processes 32-token chunks on the tensor cores (tf32 operands,
- *   fp32 accumulation and fp32 state); it needs d_k = d_v = 128, bf16 q/k/v
- *   and, for every 16 consecutive tokens and every channel, sum |g| <= 80
- *   (decay factors are formed relative to the chunk midpoint in fp32); it
- *   returns DASC_ERR_SHAPE otherwise.  AUTO picks CHUNKED when shape
- *   and dtype allow it and SEQUENTIAL when they do not.  The bound on g is
- *   checked on the device, per channel and half chunk, while the decay sums
- *   are formed: a violation is recorded in the workspace (DASC_ERR_DOMAIN
- *   from dasc_refresh_status) and the states and outputs of that call are
- *   unspecified (possibly inf or NaN); rerun it with DASC_ALGO_SEQUENTIAL.
+ *   fp32 accumulation and fp32 state); it needs d_k = d_v = 128 and bf16 q/k/v
+ *   (DASC_ERR_SHAPE otherwise) and, for every channel and every half chunk of
+ *   16 tokens, |sum g| <= 80 (decay factors are formed relative to the chunk
+ *   midpoint in fp32).  That bound is checked on the device while the sums are
+ *   formed.  A (request, layer, head) unit that breaks it is NOT written back:
+ *   its stored state keeps the bits it had before the call, its outputs are
+ *   unspecified, its index ((request*Lc + layer)*n_v_heads + head) is appended
+ *   to the int32 list that starts 256 bytes into the workspace (length: third
+ *   header word), and dasc_refresh_status reports DASC_ERR_DOMAIN.  Every other
+ *   unit is complete.
+ * algo AUTO runs CHUNKED when shape and dtype allow it, and then, on the same
+ *   stream, replays with the exact kernel (a) the units that broke the bound,
+ *   from their untouched stored states, and (b) requests of at most 8 tokens,
+ *   where one tf32-rounded q.k product can exceed the output tolerance.  Under
+ *   AUTO a call therefore completes for any g <= 0 and dasc_refresh_status
+ *   stays DASC_OK; dasc_refresh_counters tells how many units took the exact
+ *   path.  When shape or dtype rule the chunked kernel out, AUTO is SEQUENTIAL.
  *
- * workspace: DEVICE scratch of at least dasc_refresh_workspace_bytes(), 256-byte
- *   aligned, private to this call until it completes; may be NULL when that
- *   size is 0.
+ * workspace: DEVICE scratch of at least dasc_refresh_workspace_bytes() (256
+ *   bytes of flags and counters + 4 bytes per unit of the call, for CHUNKED and
+ *   AUTO), 256-byte aligned, private to this call until it completes; may be
+ *   NULL when that size is 0.
  * Errors: bad arguments -> no launch.  A bounded device-side wait that runs
- *   out, or a log-decay outside the chunked kernel's range, sets a flag in
- *   the workspace; read it with dasc_refresh_status after synchronising the
- *   stream.
+ *   out sets the first header word (DASC_ERR_TIMEOUT): the CTA that gave up
+ *   skips the rest of its work and leaves its unit's stored state untouched.
+ *   Read the flags with dasc_refresh_status after synchronising the stream.
  */
 dasc_status_t dasc_refresh_workspace_bytes(const dasc_plan_t *plan, int32_t n_req, int32_t n_layers_in_call,
                                            int32_t algo, size_t *out);
@@ -333,9 +412,20 @@ dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t l
                            size_t workspace_bytes, void *cuda_stream);
 /* After the stream has been synchronised: DASC_OK; DASC_ERR_TIMEOUT if a
  * device-side wait of the last dasc_refresh that used `workspace` gave up;
- * else DASC_ERR_DOMAIN if that call met a log-decay outside the chunked
- * kernel's range.  Copies 8 bytes device -> host (synchronous). */
+ * else DASC_ERR_DOMAIN if that call left a unit unwritten because its
+ * log-decay was outside the chunked kernel's range.  Copies the first 8
+ * bytes device -> host (synchronous); pass workspace_bytes >= 8 (with 4 only
+ * the time-out word is read).
+ * dasc_refresh_counters (same conditions, 16 bytes): units the chunked kernel
+ * handed over, and units the exact kernel replayed from that list. */
 dasc_status_t dasc_refresh_status(const void *workspace, size_t workspace_bytes);
+dasc_status_t dasc_refresh_counters(const void *workspace, size_t workspace_bytes, int32_t *handed_over,
+                                    int32_t *replayed_exactly);
+/* Test hook, not for production use: when `polls` != 0 the chunked kernel's
+ * issuing warp gives its very first wait of every CTA only that many polls, so
+ * that a test can watch a bounded wait run out (DASC_ERR_TIMEOUT, the unit left
+ * unwritten, the context still usable).  0 restores the normal limit.  Process-wide. */
+void dasc_debug_set_refresh_poll_limit(uint32_t polls);
 
 /*
  * Load path, suffix-refresh policy as the paper states it (Section 4.2, with the
@@ -379,23 +469,33 @@ dasc_status_t dasc_refresh_window(const dasc_plan_t *plan, float *state_base, in
  * back to one) can fail for lack of free memory or stall the device, and no spare buffer was
  * planned for this library.
  *
- * The kernel's scratch (its time-out flag) lives in a 4096-byte array that is part of the
- * library image: every GPU that loads libdasc holds those bytes until the process exits.  A
- * request whose scratch need (dasc_refresh_workspace_bytes) exceeds 4096 bytes is refused with
- * DASC_ERR_WORKSPACE; shapes the chunked kernel does not take get DASC_ERR_SHAPE.  The call
- * makes no cudaMalloc / cudaFree and uses no allocating library routine.
+ * The kernel's scratch lives in a 4096-byte array that is part of the library image: every
+ * GPU that loads libdasc holds those bytes until the process exits.  The first 256 bytes are
+ * the header dasc_refresh_status reads (word 0: a wait timed out; word 1: a unit outside the
+ * log-decay range was left unwritten), the remaining 3840 bytes hold the list of up to 960
+ * unit indices that the chunked kernel hands to the exact kernel for that reason.  The kernel cannot do without the header: were it ever to outgrow the array
+ * the call would return DASC_ERR_WORKSPACE; shapes the chunked kernel does not take get
+ * DASC_ERR_SHAPE.  The call makes no cudaMalloc / cudaFree and uses no allocating library
+ * routine.
  *
  * First call on a device: the library looks up the array's device address for the CURRENT
- * device (which must be the plan's device) and remembers it.  Make that first call before any
- * stream capture is begun, since the look-up is not a stream operation.
+ * device, which must be the plan's device (DASC_ERR_INVALID_ARG otherwise), and remembers it.
+ * Make that first call before any stream capture is begun, since the look-up is not a stream
+ * operation.
  * All calls on one device share the array and it keeps the last call's contents; the call
- * clears the flag on `cuda_stream` before the kernel runs.  Two dasc_refresh_static calls
- * that overlap on the GPU (different streams, no ordering) race on the flag: order them, or
- * give one of them its own workspace through dasc_refresh.
+ * clears the header words on `cuda_stream` before the kernel runs.  Two dasc_refresh_static
+ * calls that overlap on the GPU (different streams, no ordering) race on the header and the
+ * list: order them, or give one of them its own workspace through dasc_refresh.
  *
  * Arguments are those of dasc_refresh with io_dtype fixed to bf16, algo fixed to CHUNKED and
- * no workspace.  *scratch_out (may be NULL) receives the DEVICE address of the array, so that
- * after synchronising the stream dasc_refresh_status(*scratch_out, 4) reports a time-out.
+ * no workspace.  *scratch_out (may be NULL) receives the DEVICE address of the array: after
+ * synchronising the stream, dasc_refresh_status(*scratch_out, 8) reports a time-out or a
+ * log-decay outside the range (pass 8 bytes or more: with 4 only the time-out word is read).
+ * Units outside the chunked kernel's log-decay range are replayed by the exact kernel on the
+ * same stream, as under DASC_ALGO_AUTO (that kernel needs no scratch beyond the list), so the
+ * status stays DASC_OK for up to 960 such units per call; beyond that the surplus units keep
+ * their stored states and the status is DASC_ERR_DOMAIN.  Short requests are not rerouted
+ * here (algo is CHUNKED in every other respect).
  */
 dasc_status_t dasc_refresh_static(const dasc_plan_t *plan, float *state_base, int64_t layer_stride,
                                   int64_t req_stride, const int32_t *req_idx, const void *q, const void *k,

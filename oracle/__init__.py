@@ -150,6 +150,35 @@ def tp_balance(units_per_rank):
     return int(c), send
 
 
+def tp_place(packed, units_per_rank, rank, unit_words, pools):
+    """Section 4.3: put rank ``rank``'s packed slot (``U[rank]`` units) where the balanced placement wants it;
+    ``pools[s]`` is rank s's slot (numpy, 4-byte dtype, at least C units), written in place."""
+    U = np.ascontiguousarray(units_per_rank, np.int64)
+    ptrs = (C.c_void_p * U.size)(*[_words(p).ctypes.data for p in pools])
+    lib().oracle_tp_place(_p(_words(np.ascontiguousarray(packed))), _p(U), C.c_int32(U.size), C.c_int32(rank),
+                          C.c_int64(unit_words), ptrs)
+
+
+def tp_head_permutation(weight, n_ranks):
+    """Section 4.3, first stage: (perm[L][n_bundles], load[T]) for per-layer bundle weights ``weight[L][n_bundles]``."""
+    w = np.ascontiguousarray(weight, np.int64)
+    L, B = w.shape
+    assert B % n_ranks == 0
+    perm = np.full((L, B), -1, np.int32)
+    load = np.zeros(n_ranks, np.int64)
+    lib().oracle_tp_head_permutation(_p(w), C.c_int32(L), C.c_int32(B), C.c_int32(n_ranks), _p(perm), _p(load))
+    return perm, load
+
+
+def copy_blobs(src, src_stride, src_idx, dst, dst_stride, dst_idx, blob_bytes):
+    """dst[dst_idx[i]] = src[src_idx[i]] for opaque blobs (uint8 arrays, strides in bytes), in place on ``dst``."""
+    src_idx = np.ascontiguousarray(src_idx, np.int32)
+    dst_idx = np.ascontiguousarray(dst_idx, np.int32)
+    assert src.dtype == np.uint8 and dst.dtype == np.uint8
+    lib().oracle_copy_blobs(_p(src), C.c_int64(src_stride), _p(src_idx), _p(dst), C.c_int64(dst_stride), _p(dst_idx),
+                            C.c_int64(blob_bytes), C.c_int32(src_idx.size))
+
+
 def _words(a):
     assert a.dtype.itemsize == 4 and a.flags.c_contiguous
     return a.view(np.uint32)

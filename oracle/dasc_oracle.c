@@ -283,6 +283,77 @@ int64_t oracle_tp_balance(const int64_t *U, int32_t T, int64_t *send)
     return C;
 }
 
+/* Section 4.3, second stage, the placement itself: rank `rank` holds `U[rank]`
+ * packed units in `packed` (one checkpoint slot, the output of oracle_pack).
+ * Its j-th unit has global position p = U[0] + ... + U[rank-1] + j and is stored
+ * on rank p / C at local unit index p % C, C = ceil(sum U / T).  pools[s] is the
+ * slot of rank s (C units).  Walks the units one by one. */
+void oracle_tp_place(const uint32_t *packed, const int64_t *U, int32_t T, int32_t rank,
+                     int64_t unit_words, uint32_t *const *pools)
+{
+    int64_t total = 0, begin = 0;
+    for (int32_t r = 0; r < T; ++r) { total += U[r]; if (r < rank) begin += U[r]; }
+    if (total == 0) return;
+    int64_t C = (total + T - 1) / T;
+    for (int64_t j = 0; j < U[rank]; ++j) {
+        int64_t p = begin + j;
+        uint32_t *dst = pools[p / C] + (p % C) * unit_words;
+        for (int64_t w = 0; w < unit_words; ++w) dst[w] = packed[j * unit_words + w];
+    }
+}
+
+/* Section 4.3, first stage.  The paper says only that head bundles are
+ * redistributed across TP ranks at model-load time; the reading implemented:
+ * every rank keeps n_bundles / T bundles of every layer; layers are visited in
+ * ascending order and, within a layer, the not yet placed bundle with the most
+ * retained units (ties: lower index) goes to the rank whose payload so far is
+ * smallest among the ranks that still have room in this layer (ties: lower
+ * rank).  weight[l*n_bundles + b] = retained units of bundle b in layer l.
+ * perm[l*n_bundles + i] = bundle at position i; rank r owns positions
+ * [r*per, (r+1)*per) with its bundles in ascending index.  Selection by
+ * repeated scanning, no sort. */
+void oracle_tp_head_permutation(const int64_t *weight, int32_t n_layers, int32_t n_bundles,
+                                int32_t T, int32_t *perm, int64_t *load)
+{
+    int32_t per = n_bundles / T;
+    int32_t *owner = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_bundles ? n_bundles : 1));
+    int32_t *room = (int32_t *)malloc(sizeof(int32_t) * (size_t)T);
+    for (int32_t r = 0; r < T; ++r) load[r] = 0;
+    for (int32_t l = 0; l < n_layers; ++l) {
+        const int64_t *w = weight + (int64_t)l * n_bundles;
+        for (int32_t b = 0; b < n_bundles; ++b) owner[b] = -1;
+        for (int32_t r = 0; r < T; ++r) room[r] = per;
+        for (int32_t placed = 0; placed < n_bundles; ++placed) {
+            int32_t pick = -1;
+            for (int32_t b = 0; b < n_bundles; ++b)
+                if (owner[b] < 0 && (pick < 0 || w[b] > w[pick])) pick = b;
+            int32_t to = -1;
+            for (int32_t r = 0; r < T; ++r)
+                if (room[r] > 0 && (to < 0 || load[r] < load[to])) to = r;
+            owner[pick] = to;
+            room[to] -= 1;
+            load[to] += w[pick];
+        }
+        for (int32_t r = 0; r < T; ++r) {
+            int32_t i = 0;
+            for (int32_t b = 0; b < n_bundles; ++b)
+                if (owner[b] == r) perm[(int64_t)l * n_bundles + r * per + i++] = b;
+        }
+    }
+    free(owner); free(room);
+}
+
+/* The convolution state travels with a checkpoint as an opaque blob (Section
+ * 4.1): dst[dst_idx[i]] = src[src_idx[i]], blob_bytes each, strides in bytes. */
+void oracle_copy_blobs(const uint8_t *src, int64_t src_stride, const int32_t *src_idx,
+                       uint8_t *dst, int64_t dst_stride, const int32_t *dst_idx,
+                       int64_t blob_bytes, int32_t n_pairs)
+{
+    for (int32_t i = 0; i < n_pairs; ++i)
+        for (int64_t b = 0; b < blob_bytes; ++b)
+            dst[(int64_t)dst_idx[i] * dst_stride + b] = src[(int64_t)src_idx[i] * src_stride + b];
+}
+
 /* ------------------------------------------------------------------ */
 /* Store path (Section 4.1, Appendix B ragged layout): pack             */
 /* ------------------------------------------------------------------ */

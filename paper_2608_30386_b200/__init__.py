@@ -10,5 +10,6 @@ from .binding import (  # noqa: F401
     DascError, Plan, dasc_pack, dasc_plan, dasc_refresh, dasc_refresh_static, dasc_refresh_status, dasc_refresh_window, dasc_refresh_workspace_bytes,
     dasc_int8_slot_bytes, dasc_pack_int8, dasc_restore, dasc_restore_int8, lib, status_string, version,
     LAYOUT_DENSE, LAYOUT_PADDED, LAYOUT_RAGGED, dasc_checkpoint_bytes, dasc_pack_padded, dasc_padded_pool_floats,
-    dasc_restore_padded, dasc_slot_budget,
+    dasc_restore_padded, dasc_slot_budget, dasc_tp_balance, dasc_pack_tp, dasc_restore_tp, dasc_tp_head_permutation,
+    dasc_conv_store, dasc_conv_load, dasc_refresh_counters, dasc_debug_set_refresh_poll_limit,
 )

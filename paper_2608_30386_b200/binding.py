@@ -31,7 +31,8 @@ EXPORTS = (
     "dasc_plan_window", "dasc_plan_layer_counts", "dasc_plan_layer_offsets", "dasc_pack", "dasc_restore",
     "dasc_int8_slot_bytes", "dasc_pack_int8", "dasc_restore_int8",
     "dasc_padded_pool_floats", "dasc_pack_padded", "dasc_restore_padded", "dasc_checkpoint_bytes", "dasc_slot_budget",
-    "dasc_tp_balance",
+    "dasc_tp_balance", "dasc_pack_tp", "dasc_restore_tp", "dasc_tp_head_permutation", "dasc_conv_store", "dasc_conv_load",
+    "dasc_refresh_counters", "dasc_debug_set_refresh_poll_limit",
     "dasc_refresh_workspace_bytes", "dasc_refresh", "dasc_refresh_status", "dasc_refresh_window", "dasc_refresh_static",
     "dasc_status_string", "dasc_version",
 )
@@ -98,6 +99,17 @@ def lib() -> C.CDLL:
         L.dasc_checkpoint_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_int64)]
         L.dasc_slot_budget.argtypes = [C.c_int64, C.c_void_p, C.c_int32, C.c_int64, C.POINTER(C.c_int64)]
         L.dasc_tp_balance.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.c_void_p]
+        L.dasc_pack_tp.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                   C.c_int32, C.c_int32, C.c_int64, C.c_void_p, C.c_int32, C.c_void_p]
+        L.dasc_restore_tp.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int64, C.c_void_p,
+                                      C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int32, C.c_void_p]
+        L.dasc_tp_head_permutation.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.dasc_conv_store.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                      C.c_int32, C.c_void_p]
+        L.dasc_conv_load.argtypes = L.dasc_conv_store.argtypes
+        L.dasc_refresh_counters.argtypes = [C.c_void_p, C.c_size_t, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.dasc_debug_set_refresh_poll_limit.restype = None
+        L.dasc_debug_set_refresh_poll_limit.argtypes = [C.c_uint32]
         L.dasc_int8_slot_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
         L.dasc_pack_int8.argtypes = L.dasc_pack.argtypes
         L.dasc_restore_int8.argtypes = L.dasc_restore.argtypes
@@ -286,6 +298,60 @@ def dasc_tp_balance(units_per_rank):
     return int(width.value), send
 
 
+def _tp_args(pools, units_per_rank):
+    bases = (C.c_void_p * len(pools))(*[p.data_ptr() for p in pools])
+    U = np.ascontiguousarray(units_per_rank, np.int64)
+    if U.size != len(pools):
+        raise ValueError("one pool and one unit count per rank")
+    return bases, U
+
+
+def dasc_pack_tp(plan: Plan, state: torch.Tensor, layer_stride: int, req_stride: int, src_req: torch.Tensor, pools,
+                 units_per_rank, rank: int, dst_slot: torch.Tensor, slot_stride: int = 0, stream=None):
+    """Section 4.3 Store: ``dasc_pack`` with every packed unit stored straight into the pool of the rank that owns
+    its global position.  ``pools``: one device tensor per rank (this GPU's view of that rank's pool)."""
+    bases, U = _tp_args(pools, units_per_rank)
+    _check(lib().dasc_pack_tp(plan.handle, _ptr(state), layer_stride, req_stride, _ptr(src_req), bases,
+                              U.ctypes.data_as(C.c_void_p), int(U.size), int(rank), int(slot_stride), _ptr(dst_slot),
+                              int(src_req.numel()), _stream_ptr(stream)), "dasc_pack_tp")
+
+
+def dasc_restore_tp(plan: Plan, pools, units_per_rank, rank: int, src_slot: torch.Tensor, state: torch.Tensor,
+                    layer_stride: int, req_stride: int, dst_req: torch.Tensor, slot_stride: int = 0, stream=None):
+    """Section 4.3 Load: the inverse gather of ``dasc_pack_tp``, omitted units zero-filled."""
+    bases, U = _tp_args(pools, units_per_rank)
+    _check(lib().dasc_restore_tp(plan.handle, bases, U.ctypes.data_as(C.c_void_p), int(U.size), int(rank),
+                                 int(slot_stride), _ptr(src_slot), _ptr(state), layer_stride, req_stride, _ptr(dst_req),
+                                 int(src_slot.numel()), _stream_ptr(stream)), "dasc_restore_tp")
+
+
+def dasc_tp_head_permutation(plan: Plan, n_ranks: int, heads_per_bundle: int = 1):
+    """Section 4.3, first stage: (perm[L][n_bundles], units_per_rank[T]) of the load-time head-bundle placement."""
+    n_bundles = plan.info.n_v_heads // max(1, heads_per_bundle)
+    perm = np.full((plan.info.n_layers, n_bundles), -1, np.int32)
+    U = np.zeros(n_ranks, np.int64)
+    _check(lib().dasc_tp_head_permutation(plan.handle, int(n_ranks), int(heads_per_bundle),
+                                          perm.ctypes.data_as(C.c_void_p), U.ctypes.data_as(C.c_void_p)),
+           "dasc_tp_head_permutation")
+    return perm, U
+
+
+def dasc_conv_store(conv: torch.Tensor, req_stride_bytes: int, src_req: torch.Tensor, pool: torch.Tensor,
+                    slot_stride_bytes: int, dst_slot: torch.Tensor, conv_bytes: int, stream=None):
+    """Copy the convolution-state blob of each request into its checkpoint slot (Section 4.1, B_conv)."""
+    _check(lib().dasc_conv_store(_ptr(conv), int(req_stride_bytes), _ptr(src_req), _ptr(pool), int(slot_stride_bytes),
+                                 _ptr(dst_slot), int(conv_bytes), int(src_req.numel()), _stream_ptr(stream)),
+           "dasc_conv_store")
+
+
+def dasc_conv_load(pool: torch.Tensor, slot_stride_bytes: int, src_slot: torch.Tensor, conv: torch.Tensor,
+                   req_stride_bytes: int, dst_req: torch.Tensor, conv_bytes: int, stream=None):
+    """The inverse of ``dasc_conv_store``."""
+    _check(lib().dasc_conv_load(_ptr(pool), int(slot_stride_bytes), _ptr(src_slot), _ptr(conv), int(req_stride_bytes),
+                                _ptr(dst_req), int(conv_bytes), int(src_slot.numel()), _stream_ptr(stream)),
+           "dasc_conv_load")
+
+
 def dasc_int8_slot_bytes(plan: Plan) -> int:
     """Bytes of one INT8 slot: codes [packed_rows][d_v] then fp32 scales [packed_rows], rounded up to 16."""
     out = C.c_size_t()
@@ -355,10 +421,30 @@ def dasc_refresh_window(plan: Plan, state: torch.Tensor, layer_stride: int, req_
                                      _ptr(workspace), ws_bytes, _stream_ptr(stream)), "dasc_refresh_window")
 
 
-def dasc_refresh_status(workspace: torch.Tensor | None) -> int:
+def dasc_refresh_status(workspace) -> int:
+    """Status of the last refresh that used ``workspace`` (a tensor, or the device address ``dasc_refresh_static``
+    returned); call after synchronising the stream.  Reads both flag words (8 bytes)."""
     if workspace is None:
         return OK
-    return int(lib().dasc_refresh_status(_ptr(workspace), int(workspace.numel() * workspace.element_size())))
+    if isinstance(workspace, torch.Tensor):
+        return int(lib().dasc_refresh_status(_ptr(workspace), int(workspace.numel() * workspace.element_size())))
+    return int(lib().dasc_refresh_status(C.c_void_p(int(workspace)), 8))
+
+
+def dasc_refresh_counters(workspace):
+    """(units the chunked kernel handed over, units the exact kernel replayed) of the last call that used ``workspace``."""
+    a, b = C.c_int32(), C.c_int32()
+    if isinstance(workspace, torch.Tensor):
+        ptr, n = _ptr(workspace), int(workspace.numel() * workspace.element_size())
+    else:
+        ptr, n = C.c_void_p(int(workspace)), 16
+    _check(lib().dasc_refresh_counters(ptr, n, C.byref(a), C.byref(b)), "dasc_refresh_counters")
+    return int(a.value), int(b.value)
+
+
+def dasc_debug_set_refresh_poll_limit(polls: int):
+    """Test hook: poll limit of the chunked kernel's first wait (0 = normal)."""
+    lib().dasc_debug_set_refresh_poll_limit(int(polls))
 
 
 def dasc_refresh_static(plan: Plan, state: torch.Tensor, layer_stride: int, req_stride: int, req_idx: torch.Tensor,
@@ -368,8 +454,9 @@ def dasc_refresh_static(plan: Plan, state: torch.Tensor, layer_stride: int, req_
                         mode: int = REFRESH_CONTINUE, stream=None) -> int:
     """``dasc_refresh`` for callers that cannot allocate: no workspace argument, the kernel's scratch
     is a fixed array inside the library.  bf16 streams and d_k = d_v = 128 only.  Returns the device
-    address of that array (for ``dasc_refresh_status`` after a synchronise).  Calls that overlap on
-    the GPU share the array and race on its time-out flag."""
+    address of that array: pass it to ``dasc_refresh_status`` after a synchronise (both flag words are
+    read: a wait that ran out, a log-decay outside the kernel's range).  Calls that overlap on the GPU
+    share the array and race on it."""
     if q.dtype != torch.bfloat16:
         raise ValueError("dasc_refresh_static takes bf16 token streams")
     o_io = IO_BF16 if (o is not None and o.dtype == torch.bfloat16) else IO_FP32

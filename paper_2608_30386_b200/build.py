@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdasc.so")
-SOURCES = ["dasc_api.cu", "plan_host.cpp", "pack_restore.cu", "pack_restore_padded.cu", "codec_int8.cu", "refresh_seq.cu", "refresh_chunked.cu"]
+SOURCES = ["dasc_api.cu", "plan_host.cpp", "pack_restore.cu", "codec_int8.cu", "refresh_seq.cu", "refresh_chunked.cu"]
 HEADERS = [os.path.join(ROOT, "include", "dasc.h"), os.path.join(CSRC, "dasc_internal.h"),
            os.path.join(CSRC, "tcgen05_util.cuh")]
 

@@ -2,6 +2,7 @@
 // in plan_host.cpp (host plan) and in the CUDA kernels.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstring>
 #include <new>
 
@@ -46,17 +47,29 @@ void free_device_tables(dasc_plan_s *p) {
   p->d_row_keep = nullptr;
 }
 
+// The plan's index tables live on plan->info.device; a launch from another current device would hand the kernel
+// pointers of a GPU it may not be able to reach.
+dasc_status_t check_device(const dasc_plan_t *plan) {
+  if (!plan || plan->info.device < 0) return DASC_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DASC_ERR_CUDA;
+  return dev == plan->info.device ? DASC_OK : DASC_ERR_INVALID_ARG;
+}
+
 dasc_status_t check_copy_args(const dasc_plan_t *plan, const void *state, int64_t layer_stride, int64_t req_stride,
                               const void *idx_a, const void *pool, int64_t *slot_stride, const void *idx_b,
-                              int32_t n_pairs) {
+                              int32_t n_pairs, int64_t min_slot_floats = -1) {
   if (!plan) return DASC_ERR_INVALID_ARG;
   if (plan->info.device < 0) return DASC_ERR_INVALID_ARG;
   if (n_pairs < 0) return DASC_ERR_INVALID_ARG;
   if (n_pairs == 0) return DASC_OK;
   if (!state || !pool || !idx_a || !idx_b) return DASC_ERR_INVALID_ARG;
   if (!aligned16(state) || !aligned16(pool)) return DASC_ERR_INVALID_ARG;
-  if (*slot_stride == 0) *slot_stride = plan->info.slot_floats;
-  if (layer_stride < 0 || req_stride < 0 || *slot_stride < plan->info.slot_floats) return DASC_ERR_INVALID_ARG;
+  if (min_slot_floats < 0) min_slot_floats = plan->info.slot_floats;
+  if (*slot_stride == 0) *slot_stride = min_slot_floats;
+  if (layer_stride < 0 || req_stride < 0 || *slot_stride < min_slot_floats) return DASC_ERR_INVALID_ARG;
+  if (plan->info.n_layers > 65535) return DASC_ERR_SHAPE;  // one block row of the copy grids per layer
+  if (const dasc_status_t ds = check_device(plan); ds != DASC_OK) return ds;
   if (layer_stride % 4 || req_stride % 4 || *slot_stride % 4) return DASC_ERR_INVALID_ARG;
   if (plan->info.n_layers > 1 && layer_stride < plan->info.dense_floats_per_layer &&
       req_stride < plan->info.dense_floats_per_layer)
@@ -158,8 +171,8 @@ dasc_status_t dasc_pack(const dasc_plan_t *plan, const float *state_base, int64_
   dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, src_req, pool_base, &slot_stride,
                                      dst_slot, n_pairs);
   if (st != DASC_OK || n_pairs == 0) return st;
-  const int e = dasc_launch_pack(plan, state_base, layer_stride, req_stride, src_req, pool_base, slot_stride,
-                                 dst_slot, n_pairs, cuda_stream);
+  const int e = dasc_launch_pack(plan, state_base, layer_stride, req_stride, src_req, pool_base, slot_stride, 0,
+                                 dst_slot, n_pairs, 0, nullptr, cuda_stream);
   return e == 0 ? DASC_OK : DASC_ERR_CUDA;
 }
 
@@ -169,8 +182,8 @@ dasc_status_t dasc_restore(const dasc_plan_t *plan, const float *pool_base, int6
   dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, dst_req, pool_base, &slot_stride,
                                      src_slot, n_pairs);
   if (st != DASC_OK || n_pairs == 0) return st;
-  const int e = dasc_launch_restore(plan, pool_base, slot_stride, src_slot, state_base, layer_stride, req_stride,
-                                    dst_req, n_pairs, cuda_stream);
+  const int e = dasc_launch_restore(plan, pool_base, slot_stride, 0, src_slot, state_base, layer_stride, req_stride,
+                                    dst_req, n_pairs, 0, nullptr, cuda_stream);
   return e == 0 ? DASC_OK : DASC_ERR_CUDA;
 }
 
@@ -188,8 +201,8 @@ dasc_status_t dasc_pack_padded(const dasc_plan_t *plan, const float *state_base,
                                      n_pairs);
   if (st != DASC_OK || n_pairs == 0) return st;
   if (n_slots <= 0) return DASC_ERR_INVALID_ARG;
-  const int e = dasc_launch_pack_padded(plan, state_base, layer_stride, req_stride, src_req, pool_base, n_slots,
-                                        dst_slot, n_pairs, cuda_stream);
+  const int e = dasc_launch_pack(plan, state_base, layer_stride, req_stride, src_req, pool_base, 0, n_slots, dst_slot,
+                                 n_pairs, 1, nullptr, cuda_stream);
   return e == 0 ? DASC_OK : DASC_ERR_CUDA;
 }
 
@@ -201,8 +214,8 @@ dasc_status_t dasc_restore_padded(const dasc_plan_t *plan, const float *pool_bas
                                      n_pairs);
   if (st != DASC_OK || n_pairs == 0) return st;
   if (n_slots <= 0) return DASC_ERR_INVALID_ARG;
-  const int e = dasc_launch_restore_padded(plan, pool_base, n_slots, src_slot, state_base, layer_stride, req_stride,
-                                           dst_req, n_pairs, cuda_stream);
+  const int e = dasc_launch_restore(plan, pool_base, 0, n_slots, src_slot, state_base, layer_stride, req_stride,
+                                    dst_req, n_pairs, 1, nullptr, cuda_stream);
   return e == 0 ? DASC_OK : DASC_ERR_CUDA;
 }
 
@@ -256,6 +269,127 @@ dasc_status_t dasc_tp_balance(const int64_t *units_per_rank, int32_t n_ranks, in
     begin = end;
   }
   return DASC_OK;
+}
+
+dasc_status_t dasc_tp_head_permutation(const dasc_plan_t *plan, int32_t n_ranks, int32_t heads_per_bundle,
+                                       int32_t *perm, int64_t *units_per_rank) {
+  if (!plan || !perm || !units_per_rank || n_ranks <= 0 || heads_per_bundle <= 0) return DASC_ERR_INVALID_ARG;
+  const int32_t H = plan->info.n_v_heads, L = plan->info.n_layers;
+  if (H % heads_per_bundle) return DASC_ERR_INVALID_ARG;
+  const int32_t B = H / heads_per_bundle;
+  if (B % n_ranks) return DASC_ERR_INVALID_ARG;
+  const int32_t per_rank = B / n_ranks;
+  const int64_t units_per_head = plan->info.units_per_layer / H;
+  std::vector<int64_t> load(n_ranks, 0), weight(B);
+  std::vector<int32_t> order(B), room(n_ranks), owner(B);
+  for (int32_t l = 0; l < L; ++l) {
+    const uint8_t *m = plan->mask.data() + static_cast<int64_t>(l) * plan->info.units_per_layer;
+    for (int32_t b = 0; b < B; ++b) {
+      int64_t w = 0;
+      for (int64_t u = b * heads_per_bundle * units_per_head; u < (b + 1) * heads_per_bundle * units_per_head; ++u) w += m[u];
+      weight[b] = w;
+      order[b] = b;
+    }
+    // heaviest bundle first, lower index first among equals
+    std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return weight[x] > weight[y]; });
+    std::fill(room.begin(), room.end(), per_rank);
+    for (int32_t b : order) {
+      int32_t best = -1;
+      for (int32_t r = 0; r < n_ranks; ++r)
+        if (room[r] > 0 && (best < 0 || load[r] < load[best])) best = r;
+      owner[b] = best;
+      --room[best];
+      load[best] += weight[b];
+    }
+    // rank r holds positions [r * per_rank, (r + 1) * per_rank) of the permuted layer, its bundles in ascending index
+    std::vector<int32_t> fill(n_ranks, 0);
+    for (int32_t b = 0; b < B; ++b) {
+      const int32_t r = owner[b];
+      perm[static_cast<int64_t>(l) * B + r * per_rank + fill[r]++] = b;
+    }
+  }
+  for (int32_t r = 0; r < n_ranks; ++r) units_per_rank[r] = load[r];
+  return DASC_OK;
+}
+
+// Shared validation of the TP-balanced copies; fills `pl` and the slot stride.
+static dasc_status_t check_tp_args(const dasc_plan_t *plan, float *const *pool_bases, const int64_t *units_per_rank,
+                                   int32_t n_ranks, int32_t rank, int64_t *slot_stride, DascTpPlacement *pl) {
+  if (!plan || !pool_bases || !units_per_rank) return DASC_ERR_INVALID_ARG;
+  if (n_ranks <= 0 || n_ranks > DASC_TP_MAX_RANKS || rank < 0 || rank >= n_ranks) return DASC_ERR_INVALID_ARG;
+  int64_t total = 0, begin = 0;
+  for (int32_t r = 0; r < n_ranks; ++r) {
+    if (units_per_rank[r] < 0) return DASC_ERR_INVALID_ARG;
+    if (r < rank) begin += units_per_rank[r];
+    total += units_per_rank[r];
+    if (!pool_bases[r] || !aligned16(pool_bases[r])) return DASC_ERR_INVALID_ARG;
+    pl->pool_base[r] = pool_bases[r];
+  }
+  if (units_per_rank[rank] != plan->info.units_retained) return DASC_ERR_INVALID_ARG;  // U_r is this plan's payload
+  if (total >= (int64_t{1} << 31)) return DASC_ERR_SHAPE;
+  pl->n_ranks = n_ranks;
+  pl->unit_begin = begin;
+  pl->width = total > 0 ? (total + n_ranks - 1) / n_ranks : 1;
+  const int64_t min_stride = pl->width * plan->info.unit_floats;
+  if (*slot_stride == 0) *slot_stride = min_stride;
+  if (*slot_stride < min_stride || *slot_stride % 4) return DASC_ERR_INVALID_ARG;
+  return DASC_OK;
+}
+
+dasc_status_t dasc_pack_tp(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride, int64_t req_stride,
+                           const int32_t *src_req, float *const *pool_bases, const int64_t *units_per_rank,
+                           int32_t n_ranks, int32_t rank, int64_t slot_stride, const int32_t *dst_slot,
+                           int32_t n_pairs, void *cuda_stream) {
+  DascTpPlacement pl{};
+  dasc_status_t st = check_tp_args(plan, pool_bases, units_per_rank, n_ranks, rank, &slot_stride, &pl);
+  if (st != DASC_OK) return st;
+  int64_t stride_ok = slot_stride;  // the per-rank slot rule was checked above; the common rules follow
+  st = check_copy_args(plan, state_base, layer_stride, req_stride, src_req, pool_bases[0], &stride_ok, dst_slot, n_pairs, 0);
+  if (st != DASC_OK || n_pairs == 0) return st;
+  const int e = dasc_launch_pack(plan, state_base, layer_stride, req_stride, src_req, nullptr, slot_stride, 0, dst_slot,
+                                 n_pairs, 2, &pl, cuda_stream);
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+dasc_status_t dasc_restore_tp(const dasc_plan_t *plan, float *const *pool_bases, const int64_t *units_per_rank,
+                              int32_t n_ranks, int32_t rank, int64_t slot_stride, const int32_t *src_slot,
+                              float *state_base, int64_t layer_stride, int64_t req_stride, const int32_t *dst_req,
+                              int32_t n_pairs, void *cuda_stream) {
+  DascTpPlacement pl{};
+  dasc_status_t st = check_tp_args(plan, pool_bases, units_per_rank, n_ranks, rank, &slot_stride, &pl);
+  if (st != DASC_OK) return st;
+  int64_t stride_ok = slot_stride;
+  st = check_copy_args(plan, state_base, layer_stride, req_stride, dst_req, pool_bases[0], &stride_ok, src_slot, n_pairs, 0);
+  if (st != DASC_OK || n_pairs == 0) return st;
+  const int e = dasc_launch_restore(plan, nullptr, slot_stride, 0, src_slot, state_base, layer_stride, req_stride,
+                                    dst_req, n_pairs, 2, &pl, cuda_stream);
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+static dasc_status_t conv_copy(const void *src, int64_t src_stride, const int32_t *src_idx, void *dst, int64_t dst_stride,
+                               const int32_t *dst_idx, int64_t conv_bytes, int32_t n_pairs, void *cuda_stream) {
+  if (n_pairs < 0 || conv_bytes < 0) return DASC_ERR_INVALID_ARG;
+  if (n_pairs == 0 || conv_bytes == 0) return DASC_OK;
+  if (!src || !dst || !src_idx || !dst_idx || !aligned16(src) || !aligned16(dst)) return DASC_ERR_INVALID_ARG;
+  if (conv_bytes % 16 || src_stride % 16 || dst_stride % 16 || src_stride < conv_bytes || dst_stride < conv_bytes)
+    return DASC_ERR_INVALID_ARG;
+  if (conv_bytes / 16 >= (int64_t{1} << 31)) return DASC_ERR_SHAPE;
+  const int e = dasc_launch_blob_copy(src, src_stride, src_idx, dst, dst_stride, dst_idx, conv_bytes, n_pairs, cuda_stream);
+  return e == 0 ? DASC_OK : DASC_ERR_CUDA;
+}
+
+dasc_status_t dasc_conv_store(const void *conv_base, int64_t req_stride_bytes, const int32_t *src_req, void *pool_base,
+                              int64_t slot_stride_bytes, const int32_t *dst_slot, int64_t conv_bytes, int32_t n_pairs,
+                              void *cuda_stream) {
+  return conv_copy(conv_base, req_stride_bytes, src_req, pool_base, slot_stride_bytes, dst_slot, conv_bytes, n_pairs,
+                   cuda_stream);
+}
+
+dasc_status_t dasc_conv_load(const void *pool_base, int64_t slot_stride_bytes, const int32_t *src_slot, void *conv_base,
+                             int64_t req_stride_bytes, const int32_t *dst_req, int64_t conv_bytes, int32_t n_pairs,
+                             void *cuda_stream) {
+  return conv_copy(pool_base, slot_stride_bytes, src_slot, conv_base, req_stride_bytes, dst_req, conv_bytes, n_pairs,
+                   cuda_stream);
 }
 
 static int64_t int8_slot_bytes(const dasc_plan_t *plan) {
@@ -315,14 +449,24 @@ dasc_status_t dasc_refresh_workspace_bytes(const dasc_plan_t *plan, int32_t n_re
   return DASC_OK;
 }
 
+namespace {
+
+// What a validated refresh request boils down to.
+struct RefreshRequest {
+  DascRefreshArgs args{};
+  bool nothing_to_do = false;
+  bool chunked = false;  // the tensor-core kernel takes part
+  int32_t algo = DASC_ALGO_AUTO;
+};
+
+// Every argument check of dasc_refresh / dasc_refresh_window, before anything is launched.
 // tok_begin: device array of first tokens (null = cu_seqlens[r]).  q may be null when o is null.
-static dasc_status_t refresh_impl(const dasc_plan_t *plan, float *state_base, int64_t layer_stride, int64_t req_stride,
-                                  const int32_t *req_idx, const void *q, const void *k, const void *v,
-                                  int32_t io_dtype, const float *g, const float *beta, const int32_t *cu_seqlens,
-                                  const int32_t *tok_begin, int32_t n_req, int64_t total_tokens, int32_t max_seqlen,
-                                  int32_t layer_begin, int32_t layer_end, float q_scale, void *o, int32_t o_dtype,
-                                  int32_t mode, int32_t algo, void *workspace, size_t workspace_bytes,
-                                  void *cuda_stream) {
+dasc_status_t refresh_validate(const dasc_plan_t *plan, float *state_base, int64_t layer_stride, int64_t req_stride,
+                               const int32_t *req_idx, const void *q, const void *k, const void *v, int32_t io_dtype,
+                               const float *g, const float *beta, const int32_t *cu_seqlens, const int32_t *tok_begin,
+                               int32_t n_req, int64_t total_tokens, int32_t max_seqlen, int32_t layer_begin,
+                               int32_t layer_end, float q_scale, void *o, int32_t o_dtype, int32_t mode, int32_t algo,
+                               void *workspace, size_t workspace_bytes, RefreshRequest *out) {
   if (!plan || plan->info.device < 0) return DASC_ERR_INVALID_ARG;
   if (!q && !o) q = k;  // never read for its values: the kernels skip or discard the output side
   if (n_req < 0 || total_tokens < 0 || max_seqlen < 0) return DASC_ERR_INVALID_ARG;
@@ -331,7 +475,10 @@ static dasc_status_t refresh_impl(const dasc_plan_t *plan, float *state_base, in
   if (o && o_dtype != DASC_IO_BF16 && o_dtype != DASC_IO_FP32) return DASC_ERR_INVALID_ARG;
   if (mode != DASC_REFRESH_CONTINUE && mode != DASC_REFRESH_SCRATCH_MERGE_LOCAL) return DASC_ERR_INVALID_ARG;
   if (algo != DASC_ALGO_AUTO && algo != DASC_ALGO_SEQUENTIAL && algo != DASC_ALGO_CHUNKED) return DASC_ERR_INVALID_ARG;
-  if (n_req == 0 || layer_end == layer_begin || total_tokens == 0) return DASC_OK;
+  if (n_req == 0 || layer_end == layer_begin || total_tokens == 0) {
+    out->nothing_to_do = true;
+    return DASC_OK;
+  }
   if (!state_base || !req_idx || !q || !k || !v || !g || !beta || !cu_seqlens) return DASC_ERR_INVALID_ARG;
   if (!aligned16(state_base) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) ||
       (o && !aligned16(o)))
@@ -339,13 +486,15 @@ static dasc_status_t refresh_impl(const dasc_plan_t *plan, float *state_base, in
   if (layer_stride < 0 || req_stride < 0 || layer_stride % 4 || req_stride % 4) return DASC_ERR_INVALID_ARG;
   const size_t esz = io_dtype == DASC_IO_BF16 ? 2 : 4;
   if ((plan->info.d_k * esz) % 16 || (plan->info.d_v * esz) % 16) return DASC_ERR_SHAPE;
+  if (const dasc_status_t ds = check_device(plan); ds != DASC_OK) return ds;
 
   // the chunked kernel takes d_k = d_v = 128 and bf16 token streams
   const bool chunked_ok = chunked_shape_ok(plan) && io_dtype == DASC_IO_BF16;
   if (algo == DASC_ALGO_CHUNKED && !chunked_ok) return DASC_ERR_SHAPE;
-  const bool chunked = algo == DASC_ALGO_CHUNKED || (algo == DASC_ALGO_AUTO && chunked_ok);
+  out->chunked = algo == DASC_ALGO_CHUNKED || (algo == DASC_ALGO_AUTO && chunked_ok);
+  out->algo = algo;
 
-  DascRefreshArgs a{};
+  DascRefreshArgs &a = out->args;
   a.kind = plan->info.kind;
   a.H_v = plan->info.n_v_heads;
   a.H_k = plan->info.n_k_heads;
@@ -376,23 +525,43 @@ static dasc_status_t refresh_impl(const dasc_plan_t *plan, float *state_base, in
   a.rows_per_layer = plan->rows_per_layer;
   a.workspace = workspace;
   a.workspace_bytes = workspace_bytes;
-
-  int e;
-  if (chunked) {
+  a.short_thr = -1;
+  if (out->chunked) {
     const size_t need = dasc_refresh_chunked_workspace_bytes(n_req, a.n_layers_in_call, a.H_v);
-    if (need && (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u)))
-      return DASC_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return DASC_ERR_WORKSPACE;
+    a.unit_list = reinterpret_cast<int32_t *>(static_cast<unsigned char *>(workspace) + kRefreshWsHeader);
+    a.unit_list_cap = static_cast<int32_t>((need - kRefreshWsHeader) / sizeof(int32_t));
+  }
+  return DASC_OK;
+}
+
+// AUTO with a shape the tensor-core kernel takes: that kernel replays every unit inside its range and at least
+// kShortSuffix + 1 tokens long and lists the others; the exact kernel then walks the list on the same stream, from
+// stored states the first kernel has not touched.  CHUNKED runs the tensor-core kernel alone (a unit outside its
+// range is left unwritten, listed and reported); SEQUENTIAL the exact kernel alone.
+dasc_status_t refresh_launch(const RefreshRequest &rq, void *cuda_stream) {
+  if (rq.nothing_to_do) return DASC_OK;
+  DascRefreshArgs a = rq.args;
+  int e;
+  if (!rq.chunked) {
+    e = dasc_launch_refresh_seq(a, cuda_stream);
+  } else if (rq.algo == DASC_ALGO_CHUNKED) {
+    a.domain_is_error = 1;
     e = dasc_launch_refresh_chunked(a, cuda_stream);
-    if (e == -1) {
-      if (algo == DASC_ALGO_CHUNKED) return DASC_ERR_UNSUPPORTED;
+    if (e == -1) return DASC_ERR_UNSUPPORTED;
+  } else {
+    a.short_thr = kShortSuffix;
+    e = dasc_launch_refresh_chunked(a, cuda_stream);
+    if (e == 0) {
+      a.from_list = 1;
       e = dasc_launch_refresh_seq(a, cuda_stream);
     }
-  } else {
-    e = dasc_launch_refresh_seq(a, cuda_stream);
   }
   if (e == -1) return DASC_ERR_SHAPE;
   return e == 0 ? DASC_OK : DASC_ERR_CUDA;
 }
+
+}  // namespace
 
 dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t layer_stride, int64_t req_stride,
                            const int32_t *req_idx, const void *q, const void *k, const void *v, int32_t io_dtype,
@@ -401,9 +570,12 @@ dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t l
                            float q_scale, void *o, int32_t o_dtype, int32_t mode, int32_t algo, void *workspace,
                            size_t workspace_bytes, void *cuda_stream) {
   if (!q) return n_req == 0 || total_tokens == 0 || layer_end == layer_begin ? DASC_OK : DASC_ERR_INVALID_ARG;
-  return refresh_impl(plan, state_base, layer_stride, req_stride, req_idx, q, k, v, io_dtype, g, beta, cu_seqlens,
-                      nullptr, n_req, total_tokens, max_seqlen, layer_begin, layer_end, q_scale, o, o_dtype, mode, algo,
-                      workspace, workspace_bytes, cuda_stream);
+  RefreshRequest rq;
+  const dasc_status_t st = refresh_validate(plan, state_base, layer_stride, req_stride, req_idx, q, k, v, io_dtype, g,
+                                            beta, cu_seqlens, nullptr, n_req, total_tokens, max_seqlen, layer_begin,
+                                            layer_end, q_scale, o, o_dtype, mode, algo, workspace, workspace_bytes, &rq);
+  if (st != DASC_OK) return st;
+  return refresh_launch(rq, cuda_stream);
 }
 
 dasc_status_t dasc_refresh_window(const dasc_plan_t *plan, float *state_base, int64_t layer_stride,
@@ -419,22 +591,40 @@ dasc_status_t dasc_refresh_window(const dasc_plan_t *plan, float *state_base, in
   if (n_req == 0) return DASC_OK;
   if (!cu_seqlens || !window_begin) return DASC_ERR_INVALID_ARG;
   if (window > INT32_MAX) window = INT32_MAX;
+  // every check comes before the first launch: an argument error leaves window_begin untouched as well
+  RefreshRequest rq;
+  const dasc_status_t st =
+      refresh_validate(plan, state_base, layer_stride, req_stride, req_idx, q, k, v, io_dtype, g, beta, cu_seqlens,
+                       window_begin, n_req, total_tokens, static_cast<int32_t>(window), layer_begin, layer_end, q_scale, o,
+                       o_dtype, DASC_REFRESH_SCRATCH_MERGE_LOCAL, algo, workspace, workspace_bytes, &rq);
+  if (st != DASC_OK) return st;
+  if (const dasc_status_t ds = check_device(plan); ds != DASC_OK) return ds;
   window_begin_kernel<<<(n_req + 255) / 256, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(cu_seqlens, n_req, window,
                                                                                                window_begin);
   if (cudaGetLastError() != cudaSuccess) return DASC_ERR_CUDA;
   if (window == 0) return DASC_OK;  // nothing is omitted, so nothing needs a refresh
-  return refresh_impl(plan, state_base, layer_stride, req_stride, req_idx, q, k, v, io_dtype, g, beta, cu_seqlens,
-                      window_begin, n_req, total_tokens, static_cast<int32_t>(window), layer_begin, layer_end, q_scale,
-                      o, o_dtype, DASC_REFRESH_SCRATCH_MERGE_LOCAL, algo, workspace, workspace_bytes, cuda_stream);
+  return refresh_launch(rq, cuda_stream);
 }
 
 dasc_status_t dasc_refresh_status(const void *workspace, size_t workspace_bytes) {
   if (!workspace || workspace_bytes < 4) return DASC_OK;  // nothing was recorded
-  uint32_t flag[2] = {0, 0};  // [0] a wait timed out, [1] log-decay out of range
+  uint32_t flag[2] = {0, 0};  // [0] a wait timed out, [1] log-decay out of range and not replayed
   if (cudaMemcpy(flag, workspace, workspace_bytes < 8 ? 4 : 8, cudaMemcpyDeviceToHost) != cudaSuccess) return DASC_ERR_CUDA;
   if (flag[0] != 0) return DASC_ERR_TIMEOUT;
   return flag[1] == 0 ? DASC_OK : DASC_ERR_DOMAIN;
 }
+
+dasc_status_t dasc_refresh_counters(const void *workspace, size_t workspace_bytes, int32_t *handed_over,
+                                    int32_t *replayed_exactly) {
+  if (!workspace || workspace_bytes < 16 || !handed_over || !replayed_exactly) return DASC_ERR_INVALID_ARG;
+  uint32_t w[4] = {0, 0, 0, 0};
+  if (cudaMemcpy(w, workspace, 16, cudaMemcpyDeviceToHost) != cudaSuccess) return DASC_ERR_CUDA;
+  *handed_over = static_cast<int32_t>(w[2]);
+  *replayed_exactly = static_cast<int32_t>(w[3]);
+  return DASC_OK;
+}
+
+void dasc_debug_set_refresh_poll_limit(uint32_t polls) { __atomic_store_n(&g_dasc_debug_poll_limit, polls, __ATOMIC_RELAXED); }
 
 const char *dasc_status_string(dasc_status_t s) {
   switch (s) {

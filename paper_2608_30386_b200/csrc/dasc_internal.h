@@ -35,21 +35,29 @@ struct dasc_plan_s {
 // plan_host.cpp
 dasc_status_t dasc_build_plan_host(const dasc_plan_desc_t *desc, dasc_plan_s *plan);
 
-// Launchers (pack_restore.cu, refresh_seq.cu, refresh_chunked.cu).  All return cudaError_t as int.
-int dasc_launch_pack(const dasc_plan_s *plan, const float *state, int64_t layer_stride, int64_t req_stride,
-                     const int32_t *src_req, float *pool, int64_t slot_stride, const int32_t *dst_slot,
-                     int32_t n_pairs, void *stream);
-int dasc_launch_restore(const dasc_plan_s *plan, const float *pool, int64_t slot_stride, const int32_t *src_slot,
-                        float *state, int64_t layer_stride, int64_t req_stride, const int32_t *dst_req,
-                        int32_t n_pairs, void *stream);
+// Section 4.3, second stage: where this rank's packed units live in the TP group's shared storage pool.
+constexpr int DASC_TP_MAX_RANKS = 16;
+struct DascTpPlacement {
+  int32_t n_ranks;
+  float *pool_base[DASC_TP_MAX_RANKS];  // DEVICE pool of each owner rank (a peer mapping for another GPU)
+  int64_t unit_begin;                   // global position of this rank's first packed unit: sum of U_r over lower ranks
+  int64_t width;                        // C = ceil(sum_r U_r / T)
+};
 
-// pack_restore_padded.cu: pool [L][n_slots][R_max][unit]
-int dasc_launch_pack_padded(const dasc_plan_s *plan, const float *state, int64_t layer_stride, int64_t req_stride,
-                            const int32_t *src_req, float *pool, int64_t n_slots, const int32_t *dst_slot,
-                            int32_t n_pairs, void *stream);
-int dasc_launch_restore_padded(const dasc_plan_s *plan, const float *pool, int64_t n_slots, const int32_t *src_slot,
-                               float *state, int64_t layer_stride, int64_t req_stride, const int32_t *dst_req,
-                               int32_t n_pairs, void *stream);
+// Launchers (pack_restore.cu, refresh_seq.cu, refresh_chunked.cu).  All return cudaError_t as int.
+// layout: 0 ragged [slots][sum r_l] (pool_stride = floats between slots), 1 padded [L][n_slots][R_max][unit],
+// 2 TP-balanced (`placement` set; pool_stride = floats between one rank's slots).
+int dasc_launch_pack(const dasc_plan_s *plan, const float *state, int64_t layer_stride, int64_t req_stride,
+                     const int32_t *src_req, float *pool, int64_t pool_stride, int64_t n_slots, const int32_t *dst_slot,
+                     int32_t n_pairs, int layout, const DascTpPlacement *placement, void *stream);
+int dasc_launch_restore(const dasc_plan_s *plan, const float *pool, int64_t pool_stride, int64_t n_slots,
+                        const int32_t *src_slot, float *state, int64_t layer_stride, int64_t req_stride,
+                        const int32_t *dst_req, int32_t n_pairs, int layout, const DascTpPlacement *placement,
+                        void *stream);
+// dst[dst_idx[i]] = src[src_idx[i]], blobs of blob_bytes (multiple of 16)
+int dasc_launch_blob_copy(const void *src, int64_t src_stride_bytes, const int32_t *src_idx, void *dst,
+                          int64_t dst_stride_bytes, const int32_t *dst_idx, int64_t blob_bytes, int32_t n_pairs,
+                          void *stream);
 
 // codec_int8.cu
 int dasc_launch_pack_int8(const dasc_plan_s *plan, const float *state, int64_t layer_stride, int64_t req_stride,
@@ -58,6 +66,18 @@ int dasc_launch_pack_int8(const dasc_plan_s *plan, const float *state, int64_t l
 int dasc_launch_restore_int8(const dasc_plan_s *plan, const void *pool, int64_t slot_stride_bytes,
                              const int32_t *src_slot, float *state, int64_t layer_stride, int64_t req_stride,
                              const int32_t *dst_req, int32_t n_pairs, void *stream);
+
+// Refresh workspace (device): a header of 256 bytes followed by a list of unit indices.
+//   word 0  a bounded device-side wait ran out
+//   word 1  a unit left the chunked kernel's log-decay range and nothing replayed it (an error)
+//   word 2  units the chunked kernel handed over (out of range, or shorter than its threshold): length of the list
+//   word 3  units the token-by-token kernel replayed from the list
+//   bytes 256...: int32 unit indices ((request * layers_in_call + layer) * H_v + head), in hand-over order
+constexpr size_t kRefreshWsHeader = 256;
+// Requests of at most this many tokens are replayed by the exact kernel under DASC_ALGO_AUTO: with only a handful of
+// tokens every output is a sum of a few q.k products, so the tf32 rounding of one product can exceed the output
+// tolerance, and the tensor-core kernel has no speed to offer at that length anyway.
+constexpr int kShortSuffix = 8;
 
 struct DascRefreshArgs {
   int32_t kind, H_v, H_k, d_k, d_v;
@@ -79,9 +99,17 @@ struct DascRefreshArgs {
   int32_t mode;
   const uint8_t *row_keep;  // device, [L][rows_per_layer]
   int64_t rows_per_layer;
-  void *workspace;
+  void *workspace;          // header words as above (null only for the token-by-token kernel run on its own)
   size_t workspace_bytes;
+  int32_t *unit_list;       // device, or null: where units are handed over (chunked) / taken from (token-by-token)
+  int32_t unit_list_cap;    // entries the list can hold
+  int32_t short_thr;        // chunked kernel: units of at most this many tokens are handed over; -1 = none
+  int32_t from_list;        // token-by-token kernel: 1 = replay the listed units only, 0 = every unit of the grid
+  int32_t domain_is_error;  // chunked kernel: an out-of-range unit also sets word 1
+  uint32_t poll_limit_first_wait;  // test hook: poll limit of the issuing warp's very first wait (0 = the normal limit)
 };
 int dasc_launch_refresh_seq(const DascRefreshArgs &a, void *stream);
 int dasc_launch_refresh_chunked(const DascRefreshArgs &a, void *stream);
 size_t dasc_refresh_chunked_workspace_bytes(int32_t n_req, int32_t n_layers_in_call, int32_t H_v);
+// Test hook (see dasc_debug_set_refresh_poll_limit in dasc.h).
+extern uint32_t g_dasc_debug_poll_limit;

@@ -59,7 +59,7 @@ constexpr uint32_t OFF_POST = OFF_FAC + 2 * D * 4;      // [2][128] fp32 log-fac
 constexpr uint32_t OFF_BETA = OFF_POST + 2 * D * 4;     // [4][32] fp32, by chunk index mod 4 (written well ahead)
 constexpr uint32_t OFF_GSC = OFF_BETA + 4 * C * 4;      // [4][32] fp32 scalar log-decay (GDN), same ring
 constexpr uint32_t OFF_MISC = OFF_GSC + 4 * C * 4;      // barriers, tmem base, abort flag
-constexpr uint32_t SMEM_BYTES = OFF_MISC + 128;
+constexpr uint32_t SMEM_BYTES = OFF_MISC + 192;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;      // slack to align the base to 1024 bytes
 static_assert(SMEM_ALLOC <= 113 * 1024, "two CTAs per SM");
 
@@ -78,18 +78,6 @@ constexpr float kTruncComp = 1.000352f;
 constexpr float kInvTruncComp = 1.0f / kTruncComp;
 constexpr float kLog2TruncComp = 5.0774e-4f;  // log2(kTruncComp)
 
-// Development aid, compiled out by default: per-phase cycle counters of the middle CTA (chain thread 0 in slots
-// 0-10, producer thread 0 in slots 16-23), written behind the time-out flag; such a build needs 512 bytes of workspace.
-#ifdef DASC_PHASE_TIMING
-#define PT_DECL long long pt_acc[16] = {0}; long long pt_last = clock64();
-#define PT(i) do { long long pt_now = clock64(); pt_acc[i] += pt_now - pt_last; pt_last = pt_now; } while (0)
-#define PT_DUMP(who, off) do { if (blockIdx.x == gridDim.x / 2 && (who)) { long long *d = reinterpret_cast<long long *>(static_cast<char *>(a.workspace) + 64) + (off); for (int i = 0; i < 16; ++i) d[i] = pt_acc[i]; } } while (0)
-#else
-#define PT_DECL
-#define PT(i)
-#define PT_DUMP(who, off)
-#endif
-
 struct Misc {
   // tensor core -> chain warps (one tcgen05.commit each per chunk); bar_ro also releases the producer
   uint64_t bar_ap, bar_ro, bar_u, bar_o, bar_s;
@@ -105,9 +93,13 @@ struct Misc {
   uint64_t a_taken, rdy_t;
   // chain warps -> triangular warp: the T|P tile region is free again (256 arrivals per chunk)
   uint64_t tp_free;
+  // issuing thread, only after a wait has run out: arrives once every tensor-core product issued so far has completed
+  uint64_t drain;
   uint32_t tmem_base;
-  volatile uint32_t abort_flag;
+  volatile uint32_t abort_flag;   // a bounded wait ran out: every later wait of this CTA returns at once
+  volatile uint32_t domain_flag;  // a half-chunk decay sum left the range the midpoint factors can carry
 };
+static_assert(sizeof(Misc) <= 192, "Misc outgrew its shared-memory slot");
 
 __device__ __forceinline__ float ex2f(float x) {
   float y;
@@ -139,6 +131,28 @@ __device__ __forceinline__ void wait_bar(uint64_t *bar, uint32_t parity, Misc *m
     misc->abort_flag = 1;
     if (err) atomicExch(err, 1u);
   }
+}
+
+// The test hook's wait (one call site): `max_polls` non-blocking looks at the barrier, so that a short limit runs out
+// whatever the time slice of a blocking poll is.
+__device__ __forceinline__ void wait_bar_short(uint64_t *bar, uint32_t parity, Misc *misc, uint32_t *err, uint32_t max_polls) {
+  bool done = false;
+  for (uint32_t i = 0; i < max_polls && !done; ++i) done = mbar_test_wait(bar, parity);
+  if (!done) {
+    misc->abort_flag = 1;
+    if (err) atomicExch(err, 1u);
+  }
+}
+
+// This CTA does not (or could not) replay its unit: put the unit on the list that the token-by-token kernel walks
+// next on the same stream.  Without a list, or when it is full, or when the caller asked for this kernel alone, an
+// out-of-range unit is an error (word 1).
+__device__ __forceinline__ void hand_over(const DascRefreshArgs &a, bool out_of_range) {
+  uint32_t *ws = static_cast<uint32_t *>(a.workspace);
+  const uint32_t idx = atomicAdd(ws + 2, 1u);
+  const bool listed = a.unit_list && idx < static_cast<uint32_t>(a.unit_list_cap);
+  if (listed) a.unit_list[idx] = static_cast<int32_t>(blockIdx.x);
+  if (!listed || (out_of_range && a.domain_is_error)) atomicExch(ws + 1, 1u);
 }
 
 __device__ __forceinline__ void mma_tf32_16x8x8(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
@@ -229,6 +243,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   const int64_t t_begin = a.tok_begin ? a.tok_begin[r] : a.cu_seqlens[r];
   const int n_tok = static_cast<int>(a.cu_seqlens[r + 1] - t_begin);
   if (n_tok <= 0 && a.mode == DASC_REFRESH_CONTINUE) return;
+  if (n_tok <= a.short_thr) {  // left to the exact kernel (short_thr = -1: never)
+    if (tid == 0) hand_over(a, false);
+    return;
+  }
 
   float *st = a.state + static_cast<int64_t>(a.req_idx[r]) * a.req_stride + static_cast<int64_t>(layer) * a.layer_stride +
               static_cast<int64_t>(h) * D * D;
@@ -258,7 +276,9 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     mbar_init(&misc->a_taken, 32);
     mbar_init(&misc->rdy_t, 32);
     mbar_init(&misc->tp_free, NCH);
+    mbar_init(&misc->drain, 1);
     misc->abort_flag = 0;
+    misc->domain_flag = 0;
     fence_mbar_init();
   }
   if (warp == WARP_MMA) {
@@ -283,7 +303,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       // MMA1: [Kt;Qt] Kh^T.  M is padded to 128: rows 64-127 of the A tile are whatever follows it in
       // shared memory, and land in TMEM lanes 64-127 that nobody reads.
       if (lane == 0) {
-        wait_bar(&misc->rdy_prep, par, misc, err);
+        if (ch == 0 && a.poll_limit_first_wait)
+          wait_bar_short(&misc->rdy_prep, par, misc, err, a.poll_limit_first_wait);
+        else
+          wait_bar(&misc->rdy_prep, par, misc, err);
         tc_fence_after_sync();
 #pragma unroll 1
         for (int kk = 0; kk < 16; ++kk)  // K = 128 in slices of 8: block kk / 4, 32 bytes per slice inside a block
@@ -347,6 +370,13 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       }
       __syncwarp();
     }
+    // After a time-out the other roles no longer wait for the products: make sure none is still in flight when the
+    // tensor memory is given back (a real wait, bounded like the others).
+    if (lane == 0 && misc->abort_flag) {
+      mma_commit(&misc->drain);
+      mbar_wait_bounded(&misc->drain, 0, kMaxPolls);
+    }
+    __syncwarp();
   } else if (warp == WARP_T) {
     // ================================ triangular warp ================================
     // T = (I + A)^-1 depends on the token inputs only, so it is formed off the chain: A out of TMEM (lanes 0-31 are
@@ -432,7 +462,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     const int pw = warp - 8, ptid = tid - NCH;
     const int cq = lane & 7, tg = lane >> 3;
     const int c0 = pw * 32 + cq * 4;
-    PT_DECL
     // Inputs reach the producer by cp.async, each lane copying exactly the 16-byte vectors of its own tiles INTO
     // the operand tiles it will overwrite: the raw log-decay of (token t, channels c0..c0+3) lands where Kh[t][c0..]
     // goes, raw k in the first half of the Kt vector, raw q in the first half of the Qt vector.  A lane only ever
@@ -454,7 +483,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       }
       // (a) raw log-decay -> Kh tile, free once MMA1 of the previous chunk has completed
       if (ch > 0) wait_bar(&misc->bar_ap, par ^ 1, misc, err);
-      PT(0);
       if constexpr (KDA) {
 #pragma unroll
         for (int jj = 0; jj < 8; ++jj) {
@@ -467,7 +495,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       // (b) raw k, q -> Kt/Qt tile, free once MMA2 of the previous chunk has completed; by then the chain warps
       //     have also left the chunk before that one, whose parity buffers (post, Kh^T) are reused
       if (ch > 0) wait_bar(&misc->bar_ro, par ^ 1, misc, err);
-      PT(1);
 #pragma unroll
       for (int jj = 0; jj < 8; ++jj) {
         const int t = (jj >> 2) * 16 + tg * 4 + (jj & 3);
@@ -477,12 +504,9 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         if (WITH_O) cp_async8_zfill(sbase + OFF_KQ + sw128_offset(64, 32 + t, c0), gq + tt * qk_stride + c0, valid);
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
-      PT(6);
       if (!KDA) __syncwarp();  // warp 8 wrote gsc_s; the other producer warps meet it at the barrier below
       if (!KDA) asm volatile("bar.sync 2, 128;" ::: "memory");
-      PT(7);
       asm volatile("cp.async.wait_group 1;" ::: "memory");  // the log-decay has landed
-      PT(2);
       // sums: this lane's total, the prefix over the four token groups of the warp (lanes 8 apart), the half's total
       float run0[2][4], refL[4];
       bool out_of_range = false;
@@ -529,7 +553,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         }
       }
       asm volatile("cp.async.wait_group 0;" ::: "memory");  // k and q have landed
-      PT(3);
       const uint64_t l2e2 = pack2(LOG2E, LOG2E), comp2 = pack2(kLog2TruncComp, kLog2TruncComp);
       const uint64_t qs2 = pack2(a.q_scale, a.q_scale);
 #pragma unroll 1
@@ -590,13 +613,12 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           *reinterpret_cast<uint4 *>(kht_tile + sw128_offset(128, c0 + i, t4)) =
               make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
       }
-      PT(4);
-      if (out_of_range && tg == 0 && err) atomicExch(err + 1, 1u);  // the exponents of this chunk may have overflowed
+      // the exponents of this chunk may have overflowed: the unit will not be written back.  (Every lane of a channel
+      // quad holds the same totals; having only the first token group store keeps the producer loop free of spills.)
+      if (out_of_range && tg == 0) misc->domain_flag = 1;
       fence_smem_to_async();
       mbar_arrive(&misc->rdy_prep);  // -> MMA1
-      PT(5);
     }
-    PT_DUMP(ptid == 0, 16);
   } else {
     // ================================= chain warps =================================
     const int quad = warp & 3, colh = warp >> 2;                           // TMEM lane quadrant, column half
@@ -631,8 +653,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       }
       tmem_st_wait();
     }
-
-    PT_DECL
     for (int ch = 0; ch < n_chunks; ++ch) {
       const uint32_t par = ch & 1;
       const int t0 = ch * C;
@@ -643,10 +663,8 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 
       // ---- (1) the previous chunk's state update is complete; this chunk's factors and tiles are ready ----
       if (ch > 0) wait_bar(&misc->bar_s, par ^ 1, misc, err);
-      PT(0);
       wait_bar(&misc->rdy_fac[par], (ch >> 1) & 1, misc, err);
       tc_fence_after_sync();
-      PT(1);
 
       // ---- (2) state pass: thread = (value column v, half of the channels); scale the state to this chunk's midpoint ----
       {
@@ -669,7 +687,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       }
       tc_fence_before_sync();
       mbar_arrive(&misc->rdy_state);  // -> MMA2
-      PT(2);
 
       // ---- (3) P out of TMEM, by warp 1 (lanes 32-63 are its quadrant); A and T are the triangular warp's ----
       if (WITH_O && warp == 1) {
@@ -691,7 +708,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         }
         fence_smem_to_async();
       }
-      PT(3);
 
       // ---- (4) RHS^T = beta (V - R)^T as a tf32 pair: high over R^T, low in the consumed A|P columns ----
       wait_bar(&misc->bar_ro, par, misc, err);
@@ -699,7 +715,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       asm volatile("cp.async.wait_all;" ::: "memory");  // V of this chunk
       wait_bar(&misc->a_taken, par, misc, err);         // the A|P columns are about to be overwritten
       sync_chain();
-      PT(5);
       {
         const int tb = colh * 16;
         uint32_t x[16], lo[16];
@@ -721,13 +736,11 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       sync_chain();                 // everyone is done with V: the next chunk's V may land
       if (more) stage_v(ch + 1);
       asm volatile("cp.async.commit_group;" ::: "memory");
-      PT(6);
 
       // ---- (5) the part of U^T the tensor core drops when it reads it (the low 13 mantissa bits), written over
       //          the consumed RHS^T: U = U_hi + U_lo exactly ----
       wait_bar(&misc->bar_u, par, misc, err);
       tc_fence_after_sync();
-      PT(7);
       {
         const int tb = colh * 16;
         uint32_t x[16];
@@ -741,12 +754,10 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       }
       tc_fence_before_sync();
       mbar_arrive(&misc->rdy_u);  // -> MMA4, MMA5
-      PT(8);
 
       // ---- (6) outputs of this chunk ----
       wait_bar(&misc->bar_o, par, misc, err);
       tc_fence_after_sync();
-      PT(9);
       if (WITH_O) {
         const int tb = colh * 16;
         uint32_t x[16];
@@ -772,9 +783,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       tc_fence_before_sync();
       mbar_arrive(&misc->tp_free);  // this thread is done with the T|P|O tile region
       sync_chain();  // every chain thread is done with this chunk's P and O tiles before they are rewritten
-      PT(10);
     }
-    PT_DUMP(tid == 0, 0);
 
     // ---- final state: the factor still owed, then write back ----
     if (n_chunks > 0) {
@@ -785,7 +794,12 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     if (tid < D) fac_s[tid] = n_chunks > 0 ? ex2f(post_s[((n_chunks - 1) & 1) * D + tid] * LOG2E) : 1.f;
     sync_chain();
     tc_fence_after_sync();
-    {
+    // A unit whose decay left the range, or whose CTA gave up on a wait, is NOT written back: its stored state keeps
+    // the bits it had before the call, so that it can be replayed by the exact kernel (or by the caller).
+    const bool bad = misc->abort_flag != 0 || misc->domain_flag != 0;
+    if (bad) {
+      if (tid == 0 && misc->abort_flag == 0) hand_over(a, true);
+    } else {
       const uint8_t *keep = a.row_keep + static_cast<int64_t>(layer) * a.rows_per_layer + static_cast<int64_t>(h) * D;
       const bool merge = a.mode != DASC_REFRESH_CONTINUE;
 #pragma unroll 1
@@ -819,7 +833,7 @@ int launch(const DascRefreshArgs &a, void *stream) {
   const int64_t n_units = static_cast<int64_t>(a.n_req) * a.n_layers_in_call * a.H_v;
   if (n_units == 0) return cudaSuccess;
   if (n_units > 2147483647LL) return static_cast<int>(cudaErrorInvalidConfiguration);
-  e = cudaMemsetAsync(a.workspace, 0, 8, static_cast<cudaStream_t>(stream));  // clear the time-out and range flags
+  e = cudaMemsetAsync(a.workspace, 0, 16, static_cast<cudaStream_t>(stream));  // clear the four header words
   if (e != cudaSuccess) return static_cast<int>(e);
   kern<<<static_cast<unsigned>(n_units), NT, SMEM_ALLOC, static_cast<cudaStream_t>(stream)>>>(a);
   return static_cast<int>(cudaGetLastError());
@@ -827,14 +841,20 @@ int launch(const DascRefreshArgs &a, void *stream) {
 
 }  // namespace
 
-// Scratch the chunked kernel needs: a 32-bit time-out flag (first word) and a 32-bit out-of-range flag (second
-// word), padded to 256 bytes.
-size_t dasc_refresh_chunked_workspace_bytes(int32_t, int32_t, int32_t) { return 256; }
+// Scratch the chunked kernel needs: the 256-byte header (flags and counters) and one list entry per unit of the call.
+size_t dasc_refresh_chunked_workspace_bytes(int32_t n_req, int32_t n_layers_in_call, int32_t H_v) {
+  const size_t units = static_cast<size_t>(n_req) * static_cast<size_t>(n_layers_in_call) * static_cast<size_t>(H_v);
+  return kRefreshWsHeader + (units * sizeof(int32_t) + 255) / 256 * 256;
+}
+
+uint32_t g_dasc_debug_poll_limit = 0;
 
 // Returns a cudaError_t as int, or -1 if this kernel does not take the request
 // (it needs d_k = d_v = 128 and bf16 token streams).
-int dasc_launch_refresh_chunked(const DascRefreshArgs &a, void *stream) {
-  if (a.d_k != D || a.d_v != D || !a.io_bf16) return -1;
+int dasc_launch_refresh_chunked(const DascRefreshArgs &a_in, void *stream) {
+  if (a_in.d_k != D || a_in.d_v != D || !a_in.io_bf16) return -1;
+  DascRefreshArgs a = a_in;
+  a.poll_limit_first_wait = __atomic_load_n(&g_dasc_debug_poll_limit, __ATOMIC_RELAXED);
   const bool kda = a.kind == DASC_KDA;
   if (!a.o) return kda ? launch<true, __nv_bfloat16, false>(a, stream) : launch<false, __nv_bfloat16, false>(a, stream);
   if (a.o_bf16) return kda ? launch<true, __nv_bfloat16, true>(a, stream) : launch<false, __nv_bfloat16, true>(a, stream);
@@ -855,15 +875,13 @@ static __device__ __align__(256) unsigned char g_refresh_static_scratch[kStaticS
 constexpr int kMaxDevices = 64;
 void *g_static_scratch_addr[kMaxDevices] = {};  // device address per CUDA device, filled on first use
 
-// Device address of the static scratch on the CURRENT device; resolves it on the first call.
-cudaError_t static_scratch_address(void **out) {
-  int dev = -1;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
+// Device address of the static scratch on device `dev`, which must be the CURRENT device; resolves it on the
+// first call.
+cudaError_t static_scratch_address(int dev, void **out) {
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   void *p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
   if (!p) {
-    e = cudaGetSymbolAddress(&p, g_refresh_static_scratch);
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_refresh_static_scratch);
     if (e != cudaSuccess) return e;
     __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);  // racing first calls store the same value
   }
@@ -887,11 +905,16 @@ extern "C" dasc_status_t dasc_refresh_static(const dasc_plan_t *plan, float *sta
   if (o && o_dtype != DASC_IO_BF16 && o_dtype != DASC_IO_FP32) return DASC_ERR_INVALID_ARG;
   if (mode != DASC_REFRESH_CONTINUE && mode != DASC_REFRESH_SCRATCH_MERGE_LOCAL) return DASC_ERR_INVALID_ARG;
   if (plan->info.d_k != D || plan->info.d_v != D) return DASC_ERR_SHAPE;  // the chunked kernel's shape
-  // The scratch this request would need from a caller must fit the static array.
-  const size_t need = dasc_refresh_chunked_workspace_bytes(n_req, layer_end - layer_begin, plan->info.n_v_heads);
+  // The plan's tables, the caller's buffers and the scratch all have to be on the device the kernel runs on.
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return DASC_ERR_CUDA;
+  if (dev != plan->info.device) return DASC_ERR_INVALID_ARG;
+  // The scratch this kernel cannot do without (the header words) must fit the static array; the list of units left
+  // unwritten is as long as the rest of the array allows (a longer list is cut, the error word is set all the same).
+  const size_t need = kRefreshWsHeader;
   if (need > kStaticScratchBytes) return DASC_ERR_WORKSPACE;
   void *scratch = nullptr;
-  if (static_scratch_address(&scratch) != cudaSuccess) return DASC_ERR_CUDA;
+  if (static_scratch_address(dev, &scratch) != cudaSuccess) return DASC_ERR_CUDA;
   if (scratch_out) *scratch_out = scratch;
   if (n_req == 0 || layer_end == layer_begin || total_tokens == 0) return DASC_OK;
   if (!state_base || !req_idx || !q || !k || !v || !g || !beta || !cu_seqlens) return DASC_ERR_INVALID_ARG;
@@ -928,9 +951,19 @@ extern "C" dasc_status_t dasc_refresh_static(const dasc_plan_t *plan, float *sta
   a.mode = mode;
   a.row_keep = plan->d_row_keep;
   a.rows_per_layer = plan->rows_per_layer;
-  a.workspace = scratch;  // the launcher clears the time-out flag (first word) on the stream
+  a.workspace = scratch;  // the launcher clears the header words on the stream
   a.workspace_bytes = kStaticScratchBytes;
-  const int e = dasc_launch_refresh_chunked(a, cuda_stream);
+  // units outside the chunked kernel's log-decay range are listed behind the header, left unwritten, and replayed by
+  // the exact kernel right after (it needs no scratch of its own); units that do not fit the list are an error
+  a.unit_list = reinterpret_cast<int32_t *>(static_cast<unsigned char *>(scratch) + kRefreshWsHeader);
+  a.unit_list_cap = static_cast<int32_t>((kStaticScratchBytes - kRefreshWsHeader) / sizeof(int32_t));
+  a.short_thr = -1;
+  a.domain_is_error = 0;
+  int e = dasc_launch_refresh_chunked(a, cuda_stream);
   if (e == -1) return DASC_ERR_SHAPE;
+  if (e == 0) {
+    a.from_list = 1;
+    e = dasc_launch_refresh_seq(a, cuda_stream);
+  }
   return e == 0 ? DASC_OK : DASC_ERR_CUDA;
 }

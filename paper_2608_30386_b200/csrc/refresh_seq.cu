@@ -62,12 +62,12 @@ struct SeqSmem {
   float bf[TB];
 };
 
+// One (request, layer, value head) unit, replayed by the whole CTA.
 template <int DK, int DV, int RS, typename IO, typename OT, bool KDA>
-__global__ void __launch_bounds__(DV *RS) refresh_seq_kernel(DascRefreshArgs a) {
+__device__ __forceinline__ void seq_unit(const DascRefreshArgs &a, int unit, unsigned char *smem_raw) {
   constexpr int NT = DV * RS;
   constexpr int ROWS = DK / RS;  // rows of the state held by one thread
   using Smem = SeqSmem<DK, DV, IO, KDA>;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem &sm = *reinterpret_cast<Smem *>(smem_raw);
   // partial sums across row slices, double buffered by token parity
   float(*red_r)[RS][DV] = reinterpret_cast<float(*)[RS][DV]>(smem_raw + sizeof(Smem));
@@ -78,9 +78,9 @@ __global__ void __launch_bounds__(DV *RS) refresh_seq_kernel(DascRefreshArgs a) 
   const int slice = tid / DV;
   const int row0 = slice * ROWS;
 
-  const int h = blockIdx.x % a.H_v;
-  const int lc = (blockIdx.x / a.H_v) % a.n_layers_in_call;
-  const int r = blockIdx.x / (a.H_v * a.n_layers_in_call);
+  const int h = unit % a.H_v;
+  const int lc = (unit / a.H_v) % a.n_layers_in_call;
+  const int r = unit / (a.H_v * a.n_layers_in_call);
   const int hk = h / (a.H_v / a.H_k);
   const int layer = a.layer_begin + lc;
   const int64_t t_begin = a.tok_begin ? a.tok_begin[r] : a.cu_seqlens[r];
@@ -230,6 +230,25 @@ __global__ void __launch_bounds__(DV *RS) refresh_seq_kernel(DascRefreshArgs a) 
   }
 }
 
+// grid = one CTA per unit (from_list == 0), or a fixed grid whose CTAs walk the list of units that the chunked kernel
+// handed over (from_list == 1; the list and its length are in the workspace, written earlier on the same stream).
+template <int DK, int DV, int RS, typename IO, typename OT, bool KDA>
+__global__ void __launch_bounds__(DV *RS) refresh_seq_kernel(DascRefreshArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  if (!a.from_list) {
+    seq_unit<DK, DV, RS, IO, OT, KDA>(a, static_cast<int>(blockIdx.x), smem_raw);
+    return;
+  }
+  uint32_t *ws = static_cast<uint32_t *>(a.workspace);
+  const uint32_t listed = ws[2];
+  const int n_list = static_cast<int>(listed < static_cast<uint32_t>(a.unit_list_cap) ? listed : a.unit_list_cap);
+  for (int i = blockIdx.x; i < n_list; i += gridDim.x) {
+    seq_unit<DK, DV, RS, IO, OT, KDA>(a, a.unit_list[i], smem_raw);
+    if (threadIdx.x == 0) atomicAdd(ws + 3, 1u);
+    __syncthreads();  // the next unit reuses the staging buffers
+  }
+}
+
 template <int DK, int DV, int RS, typename IO, typename OT, bool KDA>
 int launch(const DascRefreshArgs &a, void *stream) {
   const size_t smem = sizeof(SeqSmem<DK, DV, IO, KDA>) + sizeof(float) * 4 * RS * DV;
@@ -239,7 +258,10 @@ int launch(const DascRefreshArgs &a, void *stream) {
   const int64_t n_units = static_cast<int64_t>(a.n_req) * a.n_layers_in_call * a.H_v;
   if (n_units == 0) return cudaSuccess;
   if (n_units > 2147483647LL) return static_cast<int>(cudaErrorInvalidConfiguration);
-  kern<<<static_cast<unsigned>(n_units), DV * RS, smem, static_cast<cudaStream_t>(stream)>>>(a);
+  // a handed-over list is short (units outside the chunked kernel's range or below its length threshold): a grid
+  // of a few CTAs per SM walks it, and costs next to nothing when the list is empty
+  const int64_t grid = a.from_list ? (n_units < 444 ? n_units : 444) : n_units;
+  kern<<<static_cast<unsigned>(grid), DV * RS, smem, static_cast<cudaStream_t>(stream)>>>(a);
   return static_cast<int>(cudaGetLastError());
 }
 

@@ -111,3 +111,112 @@ def ragged_cu_seqlens(gen, n_req: int, lo: int, hi: int) -> torch.Tensor:
 def bf16_bits(t: torch.Tensor):
     """bf16 tensor -> numpy uint16 bit patterns (CPU)."""
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view("uint16")
+
+
+@dataclass
+class TraceRound:
+    """One round of the mixed serving trace: the checkpoints stored and the cache hits served while both run."""
+    store_slots: list      # pool slot of each new checkpoint
+    hit_slots: list        # pool slot of each cache hit
+    suffix: list           # tokens since the hit checkpoint, per hit
+
+
+def serving_trace(seed: int, n_requests: int = 512, prefix_lo: int = 1024, prefix_hi: int = 131072,
+                  interval: int = 1024, n_slots: int = 2048, batch: int = 64, concurrency: int = 96,
+                  followups: int = 4, suffix_hi: int = 1024):
+    """Event list of the mixed serving trace, generated on the host from one seed.
+
+    `n_requests` requests with prefix lengths log-uniform in [prefix_lo, prefix_hi] are prefilled `concurrency` at a
+    time; a request that is picked (uniformly among the active ones) advances by `interval` tokens and stores one
+    checkpoint.  A finished request is followed up `followups` times, each after a random delay: the follow-up shares
+    a prefix of random length with it, hits the newest checkpoint at or below that length if it is still resident,
+    and replays the tokens since that checkpoint (uniform in [1, suffix_hi]).  Checkpoints live in a bounded pool of
+    `n_slots` slots recycled least-recently-used first (a store or a hit makes a slot recent); slot 0 is reserved,
+    as in the paper's allocator.  Events are cut into rounds of at most `batch` stores and `batch` hits such that no
+    hit reads a slot written in its own round and no store recycles a slot read in its own round, so the two sides
+    of a round may run concurrently.  Returns (rounds, stats)."""
+    import numpy as np
+    from collections import OrderedDict
+
+    rng = np.random.default_rng(seed)
+    prefix = np.exp(rng.uniform(math.log(prefix_lo), math.log(prefix_hi), size=n_requests)).astype(np.int64)
+    n_ckpt = prefix // interval
+    lru = OrderedDict()                      # slot -> (request, checkpoint index), least recently used first
+    where = {}                               # (request, checkpoint index) -> slot
+    free = list(range(n_slots - 1, 0, -1))   # slot 0 reserved
+    rounds, cur = [], TraceRound([], [], [])
+    written, read = set(), set()
+    stats = dict(stores=0, hits=0, misses=0, evictions=0, tokens_replayed=0, checkpoints_total=int(n_ckpt.sum()),
+                 prefix_tokens_total=int(prefix.sum()))
+
+    def close():
+        nonlocal cur, written, read
+        if cur.store_slots or cur.hit_slots:
+            rounds.append(cur)
+        cur, written, read = TraceRound([], [], []), set(), set()
+
+    def store(req, j):
+        if free:
+            slot = free.pop()
+        else:
+            slot, old = next(iter(lru.items()))
+            if slot in read or slot in written:
+                close()
+            del lru[slot]
+            del where[old]
+            stats["evictions"] += 1
+        if len(cur.store_slots) == batch:
+            close()
+        lru[slot] = (req, j)
+        where[(req, j)] = slot
+        cur.store_slots.append(slot)
+        written.add(slot)
+        stats["stores"] += 1
+
+    def hit(req):
+        shared = int(rng.integers(interval, prefix[req] + 1))          # length of the shared prefix
+        j = min(shared // interval, int(n_ckpt[req]))
+        while j >= 1 and (req, j) not in where:                        # newest resident checkpoint at or below it
+            j -= 1
+        if j < 1:
+            stats["misses"] += 1
+            return
+        slot = where[(req, j)]
+        if slot in written or len(cur.hit_slots) == batch:
+            close()
+        lru.move_to_end(slot)
+        n = int(rng.integers(1, suffix_hi + 1))
+        cur.hit_slots.append(slot)
+        cur.suffix.append(n)
+        read.add(slot)
+        stats["hits"] += 1
+        stats["tokens_replayed"] += n
+
+    nxt, active, due, clock = 0, [], [], 0       # due: (time, request) follow-ups
+    progress = {}
+    while nxt < n_requests or active or due:
+        while nxt < n_requests and len(active) < concurrency:
+            progress[nxt] = 0
+            active.append(nxt)
+            nxt += 1
+        clock += 1
+        ready = [d for d in due if d[0] <= clock]
+        if ready:
+            due = [d for d in due if d[0] > clock]
+            for _, req in ready:
+                hit(req)
+        if not active:
+            if due:
+                clock = min(d[0] for d in due) - 1
+            continue
+        req = active[int(rng.integers(0, len(active)))]
+        progress[req] += 1
+        if progress[req] <= n_ckpt[req]:
+            store(req, progress[req])
+        if progress[req] >= n_ckpt[req]:
+            active.remove(req)
+            for _ in range(followups):
+                due.append((clock + 1 + int(rng.exponential(4.0 * concurrency)), req))
+    close()
+    stats["rounds"] = len(rounds)
+    return rounds, stats

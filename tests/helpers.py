@@ -24,6 +24,49 @@ def rel_err(x, ref):
     return num / den
 
 
+def error_report(x, ref):
+    """The per-tensor metric beside two finer ones, for the log (only the first is asserted on):
+    tensor  max|x - ref| / max|ref| over the whole tensor;
+    row     the worst row of a [rows, cols] tensor taken on its own, max|x_r - ref_r| / max|ref_r| (a KDA selection
+            unit is one key-channel row of the state); rows whose reference is all zero are left out;
+    elem    max over elements of |x - ref| / max(|ref|, 1e-6 * max|ref|)."""
+    x = np.asarray(x, np.float64)
+    ref = np.asarray(ref, np.float64)
+    top = np.abs(ref).max() if ref.size else 0.0
+    if top == 0.0:
+        return {"tensor": rel_err(x, ref), "row": 0.0, "elem": 0.0}
+    err = np.abs(x - ref)
+    row_top = np.abs(ref.reshape(ref.shape[0], -1)).max(1)
+    row_err = err.reshape(ref.shape[0], -1).max(1)
+    live = row_top > 0
+    return {"tensor": float(err.max() / top), "row": float((row_err[live] / row_top[live]).max()) if live.any() else 0.0,
+            "elem": float((err / np.maximum(np.abs(ref), 1e-6 * top)).max())}
+
+
+_ERROR_LOG = {}
+
+
+def log_errors(name, kind, what, rep):
+    """Keep the worst figures per (test, kind, tensor kind); written out as JSON lines when DASC_ERROR_LOG names a file."""
+    key = (name, kind, what)
+    cur = _ERROR_LOG.setdefault(key, {"tensor": 0.0, "row": 0.0, "elem": 0.0, "units": 0})
+    for k in ("tensor", "row", "elem"):
+        cur[k] = max(cur[k], rep[k])
+    cur["units"] += 1
+
+
+def flush_error_log():
+    import json
+    import os
+    path = os.environ.get("DASC_ERROR_LOG")
+    if not path or not _ERROR_LOG:
+        return
+    with open(path, "a") as f:
+        for (name, kind, what), v in sorted(_ERROR_LOG.items()):
+            f.write(json.dumps({"test": name, "kind": "KDA" if kind == dasc.KDA else "GDN", "what": what, **v}) + "\n")
+    _ERROR_LOG.clear()
+
+
 def make_plans(kind, L, H_v, H_k, d_k, d_v, rates, *, sel, scope=dasc.SCOPE_LAYER, keep_ratio=1.0, w_max=0.0,
                device=0):
     """The library plan and the oracle plan for the same decay parameters."""
@@ -113,12 +156,20 @@ def assert_refresh_close(case: RefreshCase, got_state, got_o, ref_state, ref_o, 
             for h in range(case.H_v):
                 e = rel_err(got_state[r, l, h], ref_state[r, l, h])
                 worst = max(worst, e)
+                log_errors(_current_test(), case.kind, "state", error_report(got_state[r, l, h], ref_state[r, l, h]))
                 assert e <= tol, f"state r={r} l={l} h={h}: {e:.3e} > {tol}"
                 if got_o is not None and t1 > t0:
                     e = rel_err(got_o[l, t0:t1, h], ref_o[l, t0:t1, h])
                     worst = max(worst, e)
+                    log_errors(_current_test(), case.kind, "output", error_report(got_o[l, t0:t1, h], ref_o[l, t0:t1, h]))
                     assert e <= tol, f"o r={r} l={l} h={h}: {e:.3e} > {tol}"
+    flush_error_log()
     return worst
+
+
+def _current_test():
+    import os
+    return os.environ.get("PYTEST_CURRENT_TEST", "smoke").split(" ")[0].split("::")[-1]
 
 
 def make_refresh_case(seed, kind, L, H_v, H_k, d_k, d_v, lens, *, io_dtype=torch.bfloat16, keep_ratio=0.4,

@@ -8,7 +8,7 @@ import torch
 
 import oracle
 import paper_2608_30386_b200 as dasc
-from helpers import rel_err, stream_np
+from helpers import _current_test, error_report, flush_error_log, log_errors, rel_err, stream_np
 
 
 def sample_units(seed: int, n_req: int, n_layers: int, n_heads: int, count: int):
@@ -68,10 +68,14 @@ def check_sampled_refresh(kind, plan, oplan, state_before, state_after, layer_st
         ref_s, ref_o = oracle_one_unit(kind, H_v, H_k, s0, q, k, v, g, beta, cu, r, l, h, mode=mode, keep_rows=keep)
         e = rel_err(s1, ref_s)
         worst = max(worst, e)
+        log_errors(_current_test(), kind, "state", error_report(s1, ref_s))
         assert e <= tol, f"state of unit {(r, l, h)}: {e:.3e} > {tol}"
         if o is not None:
             t0, t1 = int(cu[r]), int(cu[r + 1])
-            e = rel_err(o[l, t0:t1, h].float().cpu().numpy(), ref_o)
+            got_o = o[l, t0:t1, h].float().cpu().numpy()
+            e = rel_err(got_o, ref_o)
             worst = max(worst, e)
+            log_errors(_current_test(), kind, "output", error_report(got_o, ref_o))
             assert e <= tol, f"output of unit {(r, l, h)}: {e:.3e} > {tol}"
+    flush_error_log()
     return worst

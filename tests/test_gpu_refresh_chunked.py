@@ -90,7 +90,7 @@ def test_log_decay_outside_the_chunked_range_is_reported():
     dev = case.state0.device
     s = case.streams
     state = case.state0.clone()
-    ws = torch.zeros(256, dtype=torch.uint8, device=dev)
+    ws = torch.zeros(dasc.dasc_refresh_workspace_bytes(case.plan, 1, 1, dasc.ALGO_CHUNKED), dtype=torch.uint8, device=dev)
     dasc.dasc_refresh(case.plan, state, 2 * 128 * 128, 2 * 128 * 128, torch.arange(1, dtype=torch.int32, device=dev),
                       s.q, s.k, s.v, s.g, s.beta, case.cu.to(dev), 64, 64, o=None, algo=dasc.ALGO_CHUNKED, workspace=ws)
     torch.cuda.synchronize()

@@ -1,4 +1,5 @@
-"""Seeded random sweep of the chunked refresh call: kinds, head groupings, ragged lengths (empty requests included),
+"""Seeded random sweep of the refresh call as a user makes it (DASC_ALGO_AUTO: the tensor-core kernel, with the exact
+kernel taking requests of a handful of tokens): kinds, head groupings, ragged lengths (empty requests included),
 both modes, with and without outputs, layer sub-ranges, a permuted request-to-state map and state strides with
 padding between requests and layers.  Every (request, layer, head) unit of every case is replayed by the fp64 oracle
 on the bits the GPU saw; guard values around each state show that nothing outside a unit is written."""
@@ -58,10 +59,10 @@ def test_random_chunked_refresh_calls(seed):
         sv[:, l * layer_stride: l * layer_stride + dense] = init[:, l].to(dev)
     before = state.clone()
     o = torch.full((Lc, max(T, 1), H_v, d), float("nan"), dtype=o_dtype, device=dev) if with_o else None
-    ws = torch.zeros(max(256, dasc.dasc_refresh_workspace_bytes(plan, n_req, Lc, dasc.ALGO_CHUNKED)), dtype=torch.uint8, device=dev)
+    ws = torch.zeros(dasc.dasc_refresh_workspace_bytes(plan, n_req, Lc, dasc.ALGO_AUTO), dtype=torch.uint8, device=dev)
     dasc.dasc_refresh(plan, state, layer_stride, req_stride, torch.from_numpy(req_idx).to(dev), q, k, v, g, beta,
                       cu.to(dev), T, max(lens), layer_begin=layer_begin, layer_end=layer_end, q_scale=q_scale, o=o,
-                      mode=mode, algo=dasc.ALGO_CHUNKED, workspace=ws)
+                      mode=mode, algo=dasc.ALGO_AUTO, workspace=ws)
     torch.cuda.synchronize()
     assert dasc.dasc_refresh_status(ws) == 0
 
@@ -98,17 +99,11 @@ def test_random_chunked_refresh_calls(seed):
                 if with_o and t1 > t0:
                     ref = ref_o
                     got = o_np[l, t0:t1, h]
-                    # An output is a dot product of a unit-norm query with a state column, so its rounding error scales
-                    # with q_scale * |column|, not with the output itself: a short scratch replay whose few q.k
-                    # products happen to cancel (seed 7 has a one-token request with |q.k| = 0.02) has outputs far
-                    # smaller than that.  The bar is therefore taken relative to the larger of max |reference| and
-                    # the magnitude a query can read from the unit's state.
-                    start = np.zeros_like(ref_s) if mode == dasc.REFRESH_SCRATCH_MERGE_LOCAL else s0.astype(np.float64)
-                    col = np.maximum(np.linalg.norm(start, axis=0), np.linalg.norm(ref_s, axis=0)).max()
-                    scale = max(np.abs(ref).max(), q_scale * col)
+                    # the stated metric, unchanged: max abs error over max |reference| of the unit's output block
+                    # (a bf16 output adds its own final rounding of up to 2^-8 of each value)
                     strict = float(np.abs(got - ref).max() / np.abs(ref).max())
                     worst_strict = max(worst_strict, strict if o_dtype == torch.float32 else 0.0)
-                    bound = TOL * scale + (np.abs(ref) * 2.0 ** -8 if o_dtype == torch.bfloat16 else 0.0)
+                    bound = TOL * np.abs(ref).max() + (np.abs(ref) * 2.0 ** -8 if o_dtype == torch.bfloat16 else 0.0)
                     bad = np.abs(got - ref) > bound
                     assert not bad.any(), (seed, r, l, h, lens, strict, np.argwhere(bad)[:4].tolist())
     # nothing outside the addressed units changed: padding, other layers, unused slots

@@ -53,7 +53,8 @@ def test_max_over_ranks_with_two_gloo_ranks():
 def test_reference_arm_runs_on_rank_zero_only():
     # under torchrun the other ranks of `--impl reference` exit 0 without work and without output
     env = dict(os.environ, RANK="1", WORLD_SIZE="2", CUDA_VISIBLE_DEVICES="")
-    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "0"],
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                        "--warmup", "0"],
                        env=env, capture_output=True, text=True, timeout=240)
     assert p.returncode == 0, p.stderr[-2000:]
     assert p.stdout.strip() == ""
@@ -110,3 +111,43 @@ def test_tp_balanced_store_and_load_exchange_two_ranks():
 
 def test_tp_balanced_store_and_load_exchange_three_ranks():
     _run_ranks(TP_WORKER.format(root=ROOT, units=[10, 1, 4]), 3)
+
+
+def test_bench_starts_its_own_ranks_when_asked_for_several_gpus():
+    # `python bench.py --gpus 2` with no launcher around it starts two ranks itself; --dry-launch makes them meet over
+    # gloo and count themselves instead of touching a GPU
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["CUDA_VISIBLE_DEVICES"] = ""
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-launch"], env=env,
+                       capture_output=True, text=True, timeout=300)
+    assert p.returncode == 0, p.stderr[-2000:]
+    line = json.loads(p.stdout.strip().splitlines()[-1])
+    assert line == {"dry_launch": True, "n_gpus": 2, "ranks": 2}
+    # a rank count that does not match --gpus is refused instead of being printed as n_gpus
+    env2 = dict(env, RANK="0", WORLD_SIZE="2", LOCAL_RANK="0", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(_free_port()))
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--dry-launch"], env=env2,
+                       capture_output=True, text=True, timeout=120)
+    assert p.returncode != 0 and "does not match" in p.stderr
+    # without GPUs the real run fails loudly, after both ranks were started
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"], env=env,
+                       capture_output=True, text=True, timeout=300)
+    assert p.returncode != 0 and "2 of 2 ranks failed" in p.stderr
+
+
+def test_serving_trace_is_seeded_bounded_and_hazard_free():
+    from paper_2608_30386_b200 import synth
+    rounds, st = synth.serving_trace(4, n_requests=64, n_slots=256, batch=16)
+    rounds2, st2 = synth.serving_trace(4, n_requests=64, n_slots=256, batch=16)
+    assert st == st2 and [r.store_slots for r in rounds] == [r.store_slots for r in rounds2]
+    assert st["stores"] == st["checkpoints_total"] and st["evictions"] > 0 and st["hits"] > 0
+    resident = {}
+    for r in rounds:
+        assert 0 < len(r.store_slots) + len(r.hit_slots) and len(r.store_slots) <= 16 and len(r.hit_slots) <= 16
+        assert len(set(r.store_slots)) == len(r.store_slots)            # distinct destination slots in one pack
+        assert not set(r.store_slots) & set(r.hit_slots)                # the two sides of a round are independent
+        assert all(0 < s < 256 for s in r.store_slots + r.hit_slots)    # slot 0 is reserved
+        assert all(s in resident for s in r.hit_slots)                  # a hit reads a slot stored in an earlier round
+        assert all(1 <= n <= 1024 for n in r.suffix) and len(r.suffix) == len(r.hit_slots)
+        for s in r.store_slots:
+            resident[s] = True

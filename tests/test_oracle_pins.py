@@ -341,6 +341,84 @@ def test_tp_balance_slot_width_and_split_counts():
     assert c == 7 and np.array_equal(send, 7 * np.eye(3, dtype=np.int64))
 
 
+def test_tp_place_hand_example_and_split_counts():
+    # Section 4.3, T = 3 ranks with U = (5, 0, 2): C = ceil(7 / 3) = 3.  Global sequence a0 a1 a2 a3 a4 c0 c1 ->
+    # rank 0 stores a0 a1 a2, rank 1 stores a3 a4 c0, rank 2 stores c1.  Only a3, a4 (to rank 1) and c0 (to rank 1)
+    # cross ranks; c1 stays on rank 2 although its global position moved.
+    U = [5, 0, 2]
+    w = 2                                                    # words per unit
+    a = np.arange(10, dtype=np.float32).reshape(5, w) + 100  # rank 0's packed units
+    c = np.arange(4, dtype=np.float32).reshape(2, w) + 200   # rank 2's packed units
+    pools = [np.full(3 * w + 1, -1, np.float32) for _ in range(3)]
+    oracle.tp_place(a, U, 0, w, pools)
+    oracle.tp_place(np.zeros(0, np.float32), U, 1, w, pools)
+    oracle.tp_place(c, U, 2, w, pools)
+    np.testing.assert_array_equal(pools[0], [100, 101, 102, 103, 104, 105, -1])
+    np.testing.assert_array_equal(pools[1], [106, 107, 108, 109, 200, 201, -1])
+    np.testing.assert_array_equal(pools[2], [202, 203, -1, -1, -1, -1, -1])
+    width, send = oracle.tp_balance(U)
+    assert width == 3
+    np.testing.assert_array_equal(send, [[3, 2, 0], [0, 0, 0], [0, 1, 1]])
+    # placing and reading back along the same rule is the identity, for random payloads
+    rng = np.random.default_rng(11)
+    for T in (2, 4, 8):
+        U = rng.integers(0, 9, size=T)
+        C = -(-int(U.sum()) // T) if U.sum() else 1
+        pools = [np.zeros(C * 3, np.float32) for _ in range(T)]
+        packed = [rng.standard_normal((u, 3)).astype(np.float32) for u in U]
+        for r in range(T):
+            oracle.tp_place(packed[r], U, r, 3, pools)
+        flat = np.concatenate(pools).reshape(-1, 3)[: int(U.sum())]      # rank order, C units each: the global sequence
+        np.testing.assert_array_equal(flat, np.concatenate(packed))
+
+
+def test_tp_head_permutation_hand_examples():
+    # Section 4.3, first stage, under the reading "heaviest bundle first to the least loaded rank that has room, every
+    # rank keeps n_bundles / T bundles per layer, payloads carry over from layer to layer".
+    # one layer, T = 2, weights 10 9 2 1: 10 -> rank 0, 9 -> rank 1, 2 -> rank 1 (9 < 10), 1 -> rank 0 (room only there)
+    perm, load = oracle.tp_head_permutation([[10, 9, 2, 1]], 2)
+    np.testing.assert_array_equal(perm, [[0, 3, 1, 2]])
+    np.testing.assert_array_equal(load, [11, 11])            # contiguous placement would give 19 and 3
+    # room bites: 8 1 1 1 with T = 2: 8 -> rank 0; 1 -> rank 1; 1 -> rank 1 (1 < 8); rank 1 is full, the last goes to rank 0
+    perm, load = oracle.tp_head_permutation([[8, 1, 1, 1]], 2)
+    np.testing.assert_array_equal(perm, [[0, 3, 1, 2]])
+    np.testing.assert_array_equal(load, [9, 2])
+    # two layers: the second layer starts from the payloads of the first (9 vs 2), so its heavy bundle goes to rank 1
+    perm, load = oracle.tp_head_permutation([[8, 1, 1, 1], [0, 0, 6, 1]], 2)
+    # 6 -> rank 1 (2 < 9): 8; 1 -> rank 1 (8 < 9): 9 and full; the two empty bundles 0, 1 go to rank 0
+    np.testing.assert_array_equal(perm[1], [0, 1, 2, 3])
+    np.testing.assert_array_equal(load, [9, 9])
+    # ties go to the lower bundle index and the lower rank: equal weights are dealt round-robin
+    perm, load = oracle.tp_head_permutation([[3, 3, 3, 3, 3, 3]], 3)
+    np.testing.assert_array_equal(perm, [[0, 3, 1, 4, 2, 5]])
+    np.testing.assert_array_equal(load, [6, 6, 6])
+    # invariants on random weights: a permutation per layer, payloads conserved, never worse than the widest bundle
+    # above the mean
+    rng = np.random.default_rng(12)
+    for T, B, L in ((2, 8, 3), (4, 8, 5), (8, 32, 4)):
+        w = rng.integers(0, 129, size=(L, B))
+        perm, load = oracle.tp_head_permutation(w, T)
+        for l in range(L):
+            assert sorted(perm[l]) == list(range(B))
+        assert load.sum() == w.sum()
+        per = B // T
+        got = np.zeros(T, np.int64)
+        for l in range(L):
+            for r in range(T):
+                got[r] += w[l, perm[l, r * per:(r + 1) * per]].sum()
+        np.testing.assert_array_equal(got, load)
+
+
+def test_copy_blobs_is_an_indexed_copy():
+    rng = np.random.default_rng(13)
+    src = rng.integers(0, 256, size=(4, 40), dtype=np.uint8)
+    dst = np.full((6, 48), 7, np.uint8)
+    oracle.copy_blobs(src, 40, [3, 1], dst, 48, [0, 5], 32)
+    want = np.full((6, 48), 7, np.uint8)
+    want[0, :32], want[5, :32] = src[3, :32], src[1, :32]
+    np.testing.assert_array_equal(dst, want)
+
+
 # ----------------------------------------------------------------------------
 # pack / restore invariants
 # ----------------------------------------------------------------------------

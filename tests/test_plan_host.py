@@ -154,3 +154,27 @@ def test_checkpoint_accounting_and_slot_budget_match_oracle_and_paper():
         dasc.dasc_checkpoint_bytes(p, 9, 0)
     with pytest.raises(dasc.DascError):
         dasc.dasc_slot_budget(100, [0, 0], 0)
+
+
+@pytest.mark.parametrize("kind,H,hpb,T", [(dasc.KDA, 8, 1, 2), (dasc.KDA, 32, 1, 8), (dasc.GDN, 32, 2, 8), (dasc.GDN, 8, 2, 4)])
+def test_head_bundle_placement_matches_oracle(kind, H, hpb, T):
+    # Section 4.3, first stage: the library's placement (sort-based) against the oracle's (scan-based) on the bundle
+    # weights of a seeded plan, and the payloads it reports against a recount from the mask
+    rng = np.random.default_rng(H * 10 + T)
+    L, d = 4, 16
+    uph = d if kind == dasc.KDA else 1
+    A_log = np.log(_rates(rng, (L, H, uph)))
+    p = dasc.dasc_plan(kind, L, H, H // hpb, d, d, A_log, np.zeros_like(A_log), sel=dasc.SEL_TOP_RATIO,
+                       scope=dasc.SCOPE_MODEL, keep_ratio=0.37, device=-1)
+    perm, U = dasc.dasc_tp_head_permutation(p, T, hpb)
+    weight = p.mask().reshape(L, H // hpb, hpb * uph).sum(-1)
+    o_perm, o_U = oracle.tp_head_permutation(weight, T)
+    np.testing.assert_array_equal(perm, o_perm)
+    np.testing.assert_array_equal(U, o_U)
+    assert U.sum() == p.units_retained
+    # the placement never leaves the heaviest rank above the contiguous split's heaviest rank on these profiles
+    per = (H // hpb) // T
+    contiguous = weight.reshape(L, T, per).sum((0, 2))
+    assert U.max() <= contiguous.max()
+    with pytest.raises(dasc.DascError):
+        dasc.dasc_tp_head_permutation(p, 3, hpb)             # bundles do not divide among 3 ranks
