@@ -47,7 +47,7 @@ constexpr uint32_t COL_S = 0, COL_AP = 128, COL_RO = 160, COL_U = 224;  // RO: R
 
 // shared memory map (bytes)
 constexpr uint32_t OFF_KQ = 0;                          // [4][64 rows][128 B]  rows 0-31 Kt, 32-63 Qt
-constexpr uint32_t OFF_KHT = OFF_KQ + 4 * 64 * 128;     // [2][128 rows][128 B] Kh^T[c][t], by chunk parity
+constexpr uint32_t OFF_KHT = OFF_KQ + 4 * 64 * 128;     // [2][4][32 rows][128 B] Kh[t][c] once more, as the MN-major operand of MMA5, by chunk parity
 constexpr uint32_t OFF_KH = OFF_KHT + 2 * 128 * 128;    // [4][32 rows][128 B]  Kh[t][c]
 constexpr uint32_t OFF_TM = OFF_KH + 4 * 32 * 128;      // [1][32 rows][128 B]  T[t][i]; TM|PM later the bf16 O tile
 constexpr uint32_t OFF_PM = OFF_TM + 32 * 128;          // [1][32 rows][128 B]  P[t][i]
@@ -294,7 +294,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 
   constexpr uint32_t ID_N32 = idesc_tf32(128, 32, false, false);
   constexpr uint32_t ID_N64 = idesc_tf32(128, 64, false, false);
-  constexpr uint32_t ID_N128 = idesc_tf32(128, 128, false, false);
+  constexpr uint32_t ID_N128_MN = idesc_tf32(128, 128, false, true);  // B = Kh[t][c]: the channel index N is the contiguous one
 
   if (warp == WARP_MMA) {
     // =========================== tensor-core issue warp ===========================
@@ -350,7 +350,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         }
 #pragma unroll 1
         for (int kk = 0; kk < 4; ++kk)
-          mma_ts(tm + COL_S, tm + COL_U + kk * 8, desc_kmajor(sbase + OFF_KHT + par * (128 * 128) + kk * 32), ID_N128, true);
+          mma_ts(tm + COL_S, tm + COL_U + kk * 8, desc_mn32(sbase + OFF_KHT + par * (128 * 128) + kk * 1024, 32 * 128), ID_N128_MN, true);
       }
       // MMA4 (low), MMA5 (low): the same with U_lo^T, which the chain warps wrote over the consumed RHS^T
       if (lane == 0) wait_bar(&misc->rdy_u, par, misc, err);
@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         mma_commit(&misc->bar_o);
 #pragma unroll 1
         for (int kk = 0; kk < 4; ++kk)
-          mma_ts(tm + COL_S, tm + COL_RO + kk * 8, desc_kmajor(sbase + OFF_KHT + par * (128 * 128) + kk * 32), ID_N128, true);
+          mma_ts(tm + COL_S, tm + COL_RO + kk * 8, desc_mn32(sbase + OFF_KHT + par * (128 * 128) + kk * 1024, 32 * 128), ID_N128_MN, true);
         mma_commit(&misc->bar_s);
       }
       __syncwarp();
@@ -561,7 +561,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         uint64_t run01 = half == 0 ? pack2(run0[0][0], run0[0][1]) : pack2(run0[1][0], run0[1][1]);
         uint64_t run23 = half == 0 ? pack2(run0[0][2], run0[0][3]) : pack2(run0[1][2], run0[1][3]);
         const uint64_t ref01 = half == 0 ? pack2(refL[0], refL[1]) : 0ull, ref23 = half == 0 ? pack2(refL[2], refL[3]) : 0ull;
-        uint32_t kht[4][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int t = t4 + j;
@@ -604,14 +603,13 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
           }
           *reinterpret_cast<uint4 *>(smem + off_k) =
               make_uint4(tf32_pre(kt[0]), tf32_pre(kt[1]), tf32_pre(kt[2]), tf32_pre(kt[3]));
-#pragma unroll
-          for (int i = 0; i < 4; ++i) kht[i][j] = tf32_pre(kh[i]);
-          *reinterpret_cast<uint4 *>(smem + off_h) = make_uint4(kht[0][j], kht[1][j], kht[2][j], kht[3][j]);
+          // Kh goes out twice, the same four values in both places: K-major (MMA1 contracts over the channels) and
+          // MN-major (MMA5 contracts over the tokens).  A tf32 MN-major operand has a swizzle of its own, so the two
+          // tiles differ in where a vector lands, not in what it holds.
+          const uint4 khv = make_uint4(tf32_pre(kh[0]), tf32_pre(kh[1]), tf32_pre(kh[2]), tf32_pre(kh[3]));
+          *reinterpret_cast<uint4 *>(smem + off_h) = khv;
+          *reinterpret_cast<uint4 *>(kht_tile + mn32_offset(32, t, c0)) = khv;
         }
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          *reinterpret_cast<uint4 *>(kht_tile + sw128_offset(128, c0 + i, t4)) =
-              make_uint4(kht[i][0], kht[i][1], kht[i][2], kht[i][3]);
       }
       // the exponents of this chunk may have overflowed: the unit will not be written back.  (Every lane of a channel
       // quad holds the same totals; having only the first token group store keeps the producer loop free of spills.)

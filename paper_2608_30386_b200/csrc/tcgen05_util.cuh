@@ -133,11 +133,27 @@ __device__ __forceinline__ uint32_t sw128_offset(uint32_t rows, uint32_t r, uint
   return blk * rows * 128u + r * 128u + ((((cin >> 2) ^ (r & 7u)) << 4) | ((cin & 3u) << 2));
 }
 
+// MN-major tf32 operand tiles (rows = K index, the M or N index contiguous along a row): the tensor core accepts one
+// swizzle for them, the 128-byte swizzle on 32-byte units.  A tile of R rows (the K index) and 32*NB tf32 columns is
+// stored as NB blocks of [R rows][128 bytes]; inside a block the 32-byte unit u of row r sits at unit position
+// u ^ (r & 3).  Blocks start 1024-byte aligned.  `col` must be a multiple of 4 (a 16-byte vector).
+__device__ __forceinline__ uint32_t mn32_offset(uint32_t rows, uint32_t r, uint32_t col) {
+  const uint32_t blk = col >> 5, cin = col & 31;
+  return blk * rows * 128u + r * 128u + ((((cin >> 3) ^ (r & 3u)) << 5) | (((cin >> 2) & 1u) << 4));
+}
+
 constexpr uint64_t kDescSw128 = (uint64_t{1} << 46) | (uint64_t{2} << 61);  // version 1, SWIZZLE_128B
 
 // K-major: 8-row groups are 1024 bytes apart (SBO); LBO is not used with swizzling.
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t smem_addr) {
   return kDescSw128 | (uint64_t{(smem_addr & 0x3FFFFu) >> 4}) | (uint64_t{1} << 16) | (uint64_t{1024 >> 4} << 32);
+}
+// MN-major, 128-byte swizzle on 32-byte units: groups of 4 K rows are 512 bytes apart (SBO), blocks of 32 elements
+// along M/N are `block_bytes` apart (LBO).  `smem_addr` points at the first K row of the slice.
+constexpr uint64_t kDescSw128Base32 = (uint64_t{1} << 46) | (uint64_t{1} << 61);  // version 1, SWIZZLE_128B_BASE32B
+__device__ __forceinline__ uint64_t desc_mn32(uint32_t smem_addr, uint32_t block_bytes) {
+  return kDescSw128Base32 | (uint64_t{(smem_addr & 0x3FFFFu) >> 4}) | (uint64_t{block_bytes >> 4} << 16) |
+         (uint64_t{512 >> 4} << 32);
 }
 // Instruction descriptor, kind::tf32, fp32 accumulation.
 __host__ __device__ constexpr uint32_t idesc_tf32(uint32_t M, uint32_t N, bool a_mn_major, bool b_mn_major) {
