@@ -22,6 +22,7 @@
 //   MMA5  S'^T      += U^T Kh     -> state    (U as a tf32 high/low pair)       tmem x smem
 // Buffers: the Kt/Qt and Kh tiles of chunk n+1 may be written once MMA2 of chunk n has completed
 // (MMA1 and MMA2 are their only readers); Kh^T, read last (MMA5), is double-buffered by chunk parity.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -95,6 +96,8 @@ struct Misc {
   uint64_t tp_free;
   // issuing thread, only after a wait has run out: arrives once every tensor-core product issued so far has completed
   uint64_t drain;
+  // TMA -> producer warps: the log-decay tile of a chunk has landed in the Kh tile (KDA)
+  uint64_t g_full;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;   // a bounded wait ran out: every later wait of this CTA returns at once
   volatile uint32_t domain_flag;  // a half-chunk decay sum left the range the midpoint factors can carry
@@ -220,7 +223,7 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
 // WITH_O = false is the state-only variant (no outputs wanted): q is never read, the Qt rows, P and the
 // output product are left out.
 template <bool KDA, typename OT, bool WITH_O>
-__global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs a) {
+__global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs a, const __grid_constant__ CUtensorMap tmap_g) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t{1023});
   const uint32_t sbase = smem_u32(smem);
@@ -253,7 +256,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   const int64_t tok0 = static_cast<int64_t>(lc) * a.total_tokens + t_begin;
   const __nv_bfloat16 *gq = static_cast<const __nv_bfloat16 *>(a.q) + (tok0 * a.H_k + hk) * D;
   const __nv_bfloat16 *gk = static_cast<const __nv_bfloat16 *>(a.k) + (tok0 * a.H_k + hk) * D;
-  const __nv_bfloat16 *gv = static_cast<const __nv_bfloat16 *>(a.v) + (tok0 * a.H_v + h) * D;
   const float *gg = a.g + (tok0 * a.H_v + h) * (KDA ? D : 1);
   const float *gb = a.beta + tok0 * a.H_v + h;
   OT *const go = WITH_O ? static_cast<OT *>(a.o) + (tok0 * a.H_v + h) * D : nullptr;
@@ -277,6 +279,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     mbar_init(&misc->rdy_t, 32);
     mbar_init(&misc->tp_free, NCH);
     mbar_init(&misc->drain, 1);
+    mbar_init(&misc->g_full, 1);
     misc->abort_flag = 0;
     misc->domain_flag = 0;
     fence_mbar_init();
@@ -315,7 +318,8 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         mma_commit(&misc->bar_ap);
       }
       __syncwarp();
-      // MMA2: S'^T [Kt;Qt]^T, the fp32 state read as a tf32 operand
+      // MMA2: S'^T [Kt;Qt]^T, the fp32 state read as a tf32 operand.  The state pass hands the channels over in two
+      // halves (each chain warp scales 32 of its 64 columns at a time): slices 0-3 and 8-11 first, then 4-7 and 12-15.
       if (lane == 0) wait_bar(&misc->rdy_state, par, misc, err);
       __syncwarp();
       if (lane == 0) {
@@ -462,10 +466,12 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     const int pw = warp - 8, ptid = tid - NCH;
     const int cq = lane & 7, tg = lane >> 3;
     const int c0 = pw * 32 + cq * 4;
-    // Inputs reach the producer by cp.async, each lane copying exactly the 16-byte vectors of its own tiles INTO
-    // the operand tiles it will overwrite: the raw log-decay of (token t, channels c0..c0+3) lands where Kh[t][c0..]
-    // goes, raw k in the first half of the Kt vector, raw q in the first half of the Qt vector.  A lane only ever
-    // reads what it copied itself, so no barrier is needed, and no register holds data in flight.
+    // Inputs land IN the operand tiles they will be overwritten with.  The raw log-decay of a chunk comes by TMA
+    // (KDA: four boxes of 32 tokens x 32 channels, 128-byte swizzle, i.e. exactly the layout of the Kh tile, so that
+    // the decay of (token t, channels c0..c0+3) sits where Kh[t][c0..] goes).  Raw k and q come by cp.async, each lane
+    // copying the 8-byte vectors of its own 4 x 4 tiles into the first half of the Kt / Qt vectors: a lane only ever
+    // reads what it copied itself, so no barrier is needed for them, and no register holds data in flight.
+    int g_issued = 0;
     float beta_next = (n_chunks > 0 && ptid < min(C, n_tok)) ? gb[ptid * b_stride] : 0.f;
     float gsc_next = (!KDA && n_chunks > 0 && ptid < min(C, n_tok)) ? gg[ptid * g_stride] : 0.f;
     for (int ch = 0; ch < n_chunks; ++ch) {
@@ -484,14 +490,16 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       // (a) raw log-decay -> Kh tile, free once MMA1 of the previous chunk has completed
       if (ch > 0) wait_bar(&misc->bar_ap, par ^ 1, misc, err);
       if constexpr (KDA) {
+        if (ptid == 0 && !misc->abort_flag) {
+          mbar_expect_tx(&misc->g_full, C * D * 4);
 #pragma unroll
-        for (int jj = 0; jj < 8; ++jj) {
-          const int t = (jj >> 2) * 16 + tg * 4 + (jj & 3);
-          const bool valid = t < ntok;
-          cp_async16_zfill(sbase + OFF_KH + sw128_offset(32, t, c0), gg + (t0 + (valid ? t : 0)) * g_stride + c0, valid);
+          for (int blk = 0; blk < 4; ++blk)
+            tma_load_3d(sbase + OFF_KH + blk * (C * 128), &tmap_g, blk * 32, h, static_cast<int32_t>(tok0 + t0), &misc->g_full);
+          ++g_issued;
         }
+      } else {
+        asm volatile("cp.async.commit_group;" ::: "memory");
       }
-      asm volatile("cp.async.commit_group;" ::: "memory");
       // (b) raw k, q -> Kt/Qt tile, free once MMA2 of the previous chunk has completed; by then the chain warps
       //     have also left the chunk before that one, whose parity buffers (post, Kh^T) are reused
       if (ch > 0) wait_bar(&misc->bar_ro, par ^ 1, misc, err);
@@ -506,7 +514,20 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       asm volatile("cp.async.commit_group;" ::: "memory");
       if (!KDA) __syncwarp();  // warp 8 wrote gsc_s; the other producer warps meet it at the barrier below
       if (!KDA) asm volatile("bar.sync 2, 128;" ::: "memory");
-      asm volatile("cp.async.wait_group 1;" ::: "memory");  // the log-decay has landed
+      if constexpr (KDA) {
+        wait_bar(&misc->g_full, par, misc, err);  // the log-decay has landed
+        if (ntok < C) {
+          // the box reached past the request's last token: those rows hold the decay of other tokens (or the
+          // zeros past the end of the stream) and are cleared, each lane its own vectors
+#pragma unroll
+          for (int jj = 0; jj < 8; ++jj) {
+            const int t = (jj >> 2) * 16 + tg * 4 + (jj & 3);
+            if (t >= ntok) *reinterpret_cast<float4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
+      } else {
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+      }
       // sums: this lane's total, the prefix over the four token groups of the warp (lanes 8 apart), the half's total
       float run0[2][4], refL[4];
       bool out_of_range = false;
@@ -617,12 +638,18 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       fence_smem_to_async();
       mbar_arrive(&misc->rdy_prep);  // -> MMA1
     }
+    // after a time-out the last log-decay copy may not have been waited for: it must have landed before the CTA leaves
+    if (KDA && ptid == 0 && misc->abort_flag && g_issued > 0) mbar_wait_bounded(&misc->g_full, (g_issued - 1) & 1, kMaxPolls);
   } else {
     // ================================= chain warps =================================
     const int quad = warp & 3, colh = warp >> 2;                           // TMEM lane quadrant, column half
     const uint32_t tlane = tm + (static_cast<uint32_t>(quad * 32) << 16);  // this warp's TMEM lanes
     const int vrow = quad * 32 + lane;                                     // the TMEM lane this thread owns
 
+    // V arrives by TMA, one box of 32 tokens x 128 values per chunk, started by one thread.  A box that reaches past
+    // the request's last token brings in the following tokens of the stream (zeros past its end): those columns are
+    // masked where V is used.
+    const __nv_bfloat16 *gv = static_cast<const __nv_bfloat16 *>(a.v) + (tok0 * a.H_v + h) * D;
     auto stage_v = [&](int ch) {
       const int t0 = ch * C, ntok = min(C, n_tok - t0);
       for (int i = tid; i < C * 16; i += NCH) {
@@ -631,11 +658,11 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         cp_async16_zfill(sbase + OFF_V + t * 256 + j * 16,
                          reinterpret_cast<const char *>(gv + (t0 + (valid ? t : 0)) * v_stride) + j * 16, valid);
       }
+      asm volatile("cp.async.commit_group;" ::: "memory");
     };
 
     if (n_chunks > 0) {
       stage_v(0);
-      asm volatile("cp.async.commit_group;" ::: "memory");
       // the start state goes into TMEM as it is; the first chunk's state pass scales it like any other
 #pragma unroll 1
       for (int c0 = colh * 64; c0 < colh * 64 + 64; c0 += 32) {
@@ -733,7 +760,6 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       mbar_arrive(&misc->rdy_rhs);  // -> MMA3 (T tile and RHS^T are ready)
       sync_chain();                 // everyone is done with V: the next chunk's V may land
       if (more) stage_v(ch + 1);
-      asm volatile("cp.async.commit_group;" ::: "memory");
 
       // ---- (5) the part of U^T the tensor core drops when it reads it (the low 13 mantissa bits), written over
       //          the consumed RHS^T: U = U_hi + U_lo exactly ----
@@ -833,7 +859,21 @@ int launch(const DascRefreshArgs &a, void *stream) {
   if (n_units > 2147483647LL) return static_cast<int>(cudaErrorInvalidConfiguration);
   e = cudaMemsetAsync(a.workspace, 0, 16, static_cast<cudaStream_t>(stream));  // clear the four header words
   if (e != cudaSuccess) return static_cast<int>(e);
-  kern<<<static_cast<unsigned>(n_units), NT, SMEM_ALLOC, static_cast<cudaStream_t>(stream)>>>(a);
+  // tensor map of the KDA log-decay [Lc*T tokens][H_v][128] fp32: boxes of 32 tokens x one head x 32 channels with the
+  // 128-byte swizzle, which is the layout of one block of the Kh operand tile (GDN has one scalar per token: no map)
+  CUtensorMap tmap_g{};
+  if (KDA) {
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(a.H_v),
+                                static_cast<cuuint64_t>(a.n_layers_in_call) * static_cast<cuuint64_t>(a.total_tokens)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * 4, static_cast<cuuint64_t>(a.H_v) * D * 4};
+    const cuuint32_t box[3] = {32, 1, static_cast<cuuint32_t>(C)};
+    const cuuint32_t ones[3] = {1, 1, 1};
+    if (cuTensorMapEncodeTiled(&tmap_g, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.g), dims, strides, box, ones,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return static_cast<int>(cudaErrorInvalidValue);
+  }
+  kern<<<static_cast<unsigned>(n_units), NT, SMEM_ALLOC, static_cast<cudaStream_t>(stream)>>>(a, tmap_g);
   return static_cast<int>(cudaGetLastError());
 }
 
