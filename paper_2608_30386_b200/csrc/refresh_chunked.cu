@@ -58,8 +58,13 @@ constexpr uint32_t OFF_X = OFF_L + C * LDX * 4;         // [32][LDX] fp32
 constexpr uint32_t OFF_FAC = OFF_X + C * LDX * 4;       // [2][128] fp32 state factor per channel, by chunk parity
 constexpr uint32_t OFF_POST = OFF_FAC + 2 * D * 4;      // [2][128] fp32 log-factor owed after a chunk, by chunk parity
 constexpr uint32_t OFF_BETA = OFF_POST + 2 * D * 4;     // [4][32] fp32, by chunk index mod 4 (written well ahead)
-constexpr uint32_t OFF_GSC = OFF_BETA + 4 * C * 4;      // [4][32] fp32 scalar log-decay (GDN), same ring
-constexpr uint32_t OFF_MISC = OFF_GSC + 4 * C * 4;      // barriers, tmem base, abort flag
+// GDN only, same ring as beta: per-token factors of the scalar decay, e1 = exp(G_t - G_m), e2 = exp(G_m - G_t)
+constexpr uint32_t OFF_E1C = OFF_BETA + 4 * C * 4;      // [4][32] fp32 e1 * (truncation compensation)
+constexpr uint32_t OFF_E2 = OFF_E1C + 4 * C * 4;        // [4][32] fp32 e2
+constexpr uint32_t OFF_BTE1 = OFF_E2 + 4 * C * 4;       // [4][32] fp32 beta * e1
+constexpr uint32_t OFF_MISC = OFF_BTE1 + 4 * C * 4;     // barriers, tmem base, abort flag
+// GDN only: raw k (rows 0-31) and q (rows 32-63) as bf16, [2][64 rows][128 B], in the place of the K-major Kh tile
+constexpr uint32_t OFF_KQ16 = OFF_KH;
 constexpr uint32_t SMEM_BYTES = OFF_MISC + 192;
 constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;      // slack to align the base to 1024 bytes
 static_assert(SMEM_ALLOC <= 113 * 1024, "two CTAs per SM");
@@ -232,7 +237,9 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   float *fac_s = reinterpret_cast<float *>(smem + OFF_FAC);
   float *post_s = reinterpret_cast<float *>(smem + OFF_POST);
   float *beta_s = reinterpret_cast<float *>(smem + OFF_BETA);
-  float *gsc_s = reinterpret_cast<float *>(smem + OFF_GSC);
+  float *e1c_s = reinterpret_cast<float *>(smem + OFF_E1C);
+  float *e2_s = reinterpret_cast<float *>(smem + OFF_E2);
+  float *bte1_s = reinterpret_cast<float *>(smem + OFF_BTE1);
   const __nv_bfloat16 *Vs = reinterpret_cast<const __nv_bfloat16 *>(smem + OFF_V);
   Misc *misc = reinterpret_cast<Misc *>(smem + OFF_MISC);
   uint32_t *err = static_cast<uint32_t *>(a.workspace);
@@ -296,6 +303,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   constexpr float LOG2E = 1.4426950408889634f;
 
   constexpr uint32_t ID_N32 = idesc_tf32(128, 32, false, false);
+  constexpr uint32_t ID_BF16_N32 = idesc_bf16(128, 32);
   constexpr uint32_t ID_N64 = idesc_tf32(128, 64, false, false);
   constexpr uint32_t ID_N128_MN = idesc_tf32(128, 128, false, true);  // B = Kh[t][c]: the channel index N is the contiguous one
 
@@ -311,10 +319,21 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         else
           wait_bar(&misc->rdy_prep, par, misc, err);
         tc_fence_after_sync();
+        if constexpr (KDA) {
 #pragma unroll 1
-        for (int kk = 0; kk < 16; ++kk)  // K = 128 in slices of 8: block kk / 4, 32 bytes per slice inside a block
-          mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
-                 desc_kmajor(sbase + OFF_KH + (kk >> 2) * (32 * 128) + (kk & 3) * 32), ID_N32, kk != 0);
+          for (int kk = 0; kk < 16; ++kk)  // K = 128 in slices of 8: block kk / 4, 32 bytes per slice inside a block
+            mma_ss(tm + COL_AP, desc_kmajor(sbase + OFF_KQ + (kk >> 2) * (64 * 128) + (kk & 3) * 32),
+                   desc_kmajor(sbase + OFF_KH + (kk >> 2) * (32 * 128) + (kk & 3) * 32), ID_N32, kk != 0);
+        } else {
+          // GDN: the decay is one scalar per token, so it is applied to A and P after the product, and the product
+          // itself is [k; q] k^T on the raw bf16 inputs: exact operands, K = 16 per instruction.  A and B come from
+          // the same tile (B = its first 32 rows).
+#pragma unroll 1
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t d = desc_kmajor(sbase + OFF_KQ16 + (kk >> 2) * (64 * 128) + (kk & 3) * 32);
+            mma_ss_bf16(tm + COL_AP, d, d, ID_BF16_N32, kk != 0);
+          }
+        }
         mma_commit(&misc->bar_ap);
       }
       __syncwarp();
@@ -398,14 +417,18 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       mbar_arrive(&misc->a_taken);  // the chain warps may reuse the A|P columns
       const int t = lane;
       // row t of A = strict_lower(Kt Kh^T) * beta_t, kept in fp32 for the inverse
-      const float bt = beta_c[t] * kInvTruncComp;
+      // KDA: the decay is inside the product, whose Kt rows carry the truncation compensation.  GDN: the product is
+      // the raw k_t . k_j and the decay exp(G_t - G_j) = e1_t e2_j is applied here.
+      const float bt = KDA ? beta_c[t] * kInvTruncComp : bte1_s[(ch & 3) * C + t];
 #pragma unroll
       for (int j = 0; j < 32; j += 4) {
+        float4 e2 = make_float4(1.f, 1.f, 1.f, 1.f);
+        if constexpr (!KDA) e2 = *reinterpret_cast<const float4 *>(e2_s + (ch & 3) * C + j);
         float4 o;
-        o.x = (j + 0 < t) ? bt * __uint_as_float(x[j + 0]) : 0.f;
-        o.y = (j + 1 < t) ? bt * __uint_as_float(x[j + 1]) : 0.f;
-        o.z = (j + 2 < t) ? bt * __uint_as_float(x[j + 2]) : 0.f;
-        o.w = (j + 3 < t) ? bt * __uint_as_float(x[j + 3]) : 0.f;
+        o.x = (j + 0 < t) ? bt * e2.x * __uint_as_float(x[j + 0]) : 0.f;
+        o.y = (j + 1 < t) ? bt * e2.y * __uint_as_float(x[j + 1]) : 0.f;
+        o.z = (j + 2 < t) ? bt * e2.z * __uint_as_float(x[j + 2]) : 0.f;
+        o.w = (j + 3 < t) ? bt * e2.w * __uint_as_float(x[j + 3]) : 0.f;
         *reinterpret_cast<float4 *>(Lm + t * LDX + j) = o;
       }
       __syncwarp();
@@ -474,6 +497,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
     int g_issued = 0;
     float beta_next = (n_chunks > 0 && ptid < min(C, n_tok)) ? gb[ptid * b_stride] : 0.f;
     float gsc_next = (!KDA && n_chunks > 0 && ptid < min(C, n_tok)) ? gg[ptid * g_stride] : 0.f;
+    float gsc_cur = 0.f, post_prev = 0.f;  // GDN, first producer warp: this chunk's log-decay, the factor owed by the previous chunk
     for (int ch = 0; ch < n_chunks; ++ch) {
       const uint32_t par = ch & 1;
       const int t0 = ch * C, ntok = min(C, n_tok - t0);
@@ -482,7 +506,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
       // the next chunk's are fetched now and stored one iteration later
       if (ptid < C) {
         beta_s[(ch & 3) * C + ptid] = beta_next;
-        if (!KDA) gsc_s[(ch & 3) * C + ptid] = gsc_next;
+        if (!KDA) gsc_cur = gsc_next;
         const bool v1 = ch + 1 < n_chunks && ptid < min(C, n_tok - t0 - C);
         beta_next = v1 ? gb[(t0 + C + ptid) * b_stride] : 0.f;
         if (!KDA) gsc_next = v1 ? gg[(t0 + C + ptid) * g_stride] : 0.f;
@@ -512,129 +536,170 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         if (WITH_O) cp_async8_zfill(sbase + OFF_KQ + sw128_offset(64, 32 + t, c0), gq + tt * qk_stride + c0, valid);
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
-      if (!KDA) __syncwarp();  // warp 8 wrote gsc_s; the other producer warps meet it at the barrier below
-      if (!KDA) asm volatile("bar.sync 2, 128;" ::: "memory");
       if constexpr (KDA) {
-        wait_bar(&misc->g_full, par, misc, err);  // the log-decay has landed
-        if (ntok < C) {
-          // the box reached past the request's last token: those rows hold the decay of other tokens (or the
-          // zeros past the end of the stream) and are cleared, each lane its own vectors
-#pragma unroll
-          for (int jj = 0; jj < 8; ++jj) {
-            const int t = (jj >> 2) * 16 + tg * 4 + (jj & 3);
-            if (t >= ntok) *reinterpret_cast<float4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_float4(0.f, 0.f, 0.f, 0.f);
+        {
+          wait_bar(&misc->g_full, par, misc, err);  // the log-decay has landed
+          if (ntok < C) {
+            // the box reached past the request's last token: those rows hold the decay of other tokens (or the
+            // zeros past the end of the stream) and are cleared, each lane its own vectors
+  #pragma unroll
+            for (int jj = 0; jj < 8; ++jj) {
+              const int t = (jj >> 2) * 16 + tg * 4 + (jj & 3);
+              if (t >= ntok) *reinterpret_cast<float4 *>(smem + OFF_KH + sw128_offset(32, t, c0)) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
           }
         }
-      } else {
-        asm volatile("cp.async.wait_group 1;" ::: "memory");
-      }
-      // sums: this lane's total, the prefix over the four token groups of the warp (lanes 8 apart), the half's total
-      float run0[2][4], refL[4];
-      bool out_of_range = false;
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        float own[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int t = half * 16 + tg * 4 + j;
-          if constexpr (KDA) {
+        // sums: this lane's total, the prefix over the four token groups of the warp (lanes 8 apart), the half's total
+        float run0[2][4], refL[4];
+        bool out_of_range = false;
+  #pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          float own[4] = {0.f, 0.f, 0.f, 0.f};
+  #pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int t = half * 16 + tg * 4 + j;
             const float4 g4 = *reinterpret_cast<const float4 *>(smem + OFF_KH + sw128_offset(32, t, c0));
             own[0] += g4.x; own[1] += g4.y; own[2] += g4.z; own[3] += g4.w;
-          } else {
-            const float gs = gsc_s[(ch & 3) * C + t];
-            own[0] += gs; own[1] += gs; own[2] += gs; own[3] += gs;
+          }
+          float tot[4];
+  #pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float incl = own[i];
+            float x = __shfl_up_sync(0xffffffffu, incl, 8);
+            if (tg >= 1) incl += x;
+            x = __shfl_up_sync(0xffffffffu, incl, 16);
+            if (tg >= 2) incl += x;
+            run0[half][i] = incl - own[i];                      // accumulated before this lane's first token
+            tot[i] = __shfl_sync(0xffffffffu, incl, cq + 24);    // the half's total
+            if (half == 0) refL[i] = -tot[i] * LOG2E;            // minus the midpoint reference, in log2 units
+            out_of_range |= !(fabsf(tot[i]) <= kMaxHalfDecay);   // also true for NaN
+          }
+          if (half == 0) {
+            // The factor that takes the state from where the previous chunk left it to this chunk's midpoint needs
+            // the first half's sums only: it is handed to the chain warps before the tiles are built.
+            if (tg == 0) {
+              const float4 post_prev = ch > 0 ? *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0)
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+              *reinterpret_cast<float4 *>(fac_s + par * D + c0) =
+                  make_float4(ex2f((post_prev.x + tot[0]) * LOG2E), ex2f((post_prev.y + tot[1]) * LOG2E),
+                              ex2f((post_prev.z + tot[2]) * LOG2E), ex2f((post_prev.w + tot[3]) * LOG2E));
+            }
+            mbar_arrive(&misc->rdy_fac[par]);
+          } else if (tg == 0) {
+            *reinterpret_cast<float4 *>(post_s + par * D + c0) = make_float4(tot[0], tot[1], tot[2], tot[3]);  // G_C - G_m
           }
         }
-        float tot[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          float incl = own[i];
-          float x = __shfl_up_sync(0xffffffffu, incl, 8);
-          if (tg >= 1) incl += x;
-          x = __shfl_up_sync(0xffffffffu, incl, 16);
-          if (tg >= 2) incl += x;
-          run0[half][i] = incl - own[i];                      // accumulated before this lane's first token
-          tot[i] = __shfl_sync(0xffffffffu, incl, cq + 24);    // the half's total
-          if (half == 0) refL[i] = -tot[i] * LOG2E;            // minus the midpoint reference, in log2 units
-          out_of_range |= !(fabsf(tot[i]) <= kMaxHalfDecay);   // also true for NaN
-        }
-        if (half == 0) {
-          // The factor that takes the state from where the previous chunk left it to this chunk's midpoint needs
-          // the first half's sums only: it is handed to the chain warps before the tiles are built.
-          if (tg == 0) {
-            const float4 post_prev = ch > 0 ? *reinterpret_cast<const float4 *>(post_s + (par ^ 1) * D + c0)
-                                            : make_float4(0.f, 0.f, 0.f, 0.f);
-            *reinterpret_cast<float4 *>(fac_s + par * D + c0) =
-                make_float4(ex2f((post_prev.x + tot[0]) * LOG2E), ex2f((post_prev.y + tot[1]) * LOG2E),
-                            ex2f((post_prev.z + tot[2]) * LOG2E), ex2f((post_prev.w + tot[3]) * LOG2E));
-          }
-          mbar_arrive(&misc->rdy_fac[par]);
-        } else if (tg == 0) {
-          *reinterpret_cast<float4 *>(post_s + par * D + c0) = make_float4(tot[0], tot[1], tot[2], tot[3]);  // G_C - G_m
-        }
-      }
-      asm volatile("cp.async.wait_group 0;" ::: "memory");  // k and q have landed
-      const uint64_t l2e2 = pack2(LOG2E, LOG2E), comp2 = pack2(kLog2TruncComp, kLog2TruncComp);
-      const uint64_t qs2 = pack2(a.q_scale, a.q_scale);
-#pragma unroll 1
-      for (int half = 0; half < 2; ++half) {
-        const int t4 = half * 16 + tg * 4;
-        uint64_t run01 = half == 0 ? pack2(run0[0][0], run0[0][1]) : pack2(run0[1][0], run0[1][1]);
-        uint64_t run23 = half == 0 ? pack2(run0[0][2], run0[0][3]) : pack2(run0[1][2], run0[1][3]);
-        const uint64_t ref01 = half == 0 ? pack2(refL[0], refL[1]) : 0ull, ref23 = half == 0 ? pack2(refL[2], refL[3]) : 0ull;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int t = t4 + j;
-          const uint32_t off_k = OFF_KQ + sw128_offset(64, t, c0), off_q = OFF_KQ + sw128_offset(64, 32 + t, c0);
-          const uint32_t off_h = OFF_KH + sw128_offset(32, t, c0);
-          const uint2 kw = *reinterpret_cast<const uint2 *>(smem + off_k);
-          uint64_t g01, g23;
-          if constexpr (KDA) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");  // k and q have landed
+        const uint64_t l2e2 = pack2(LOG2E, LOG2E), comp2 = pack2(kLog2TruncComp, kLog2TruncComp);
+        const uint64_t qs2 = pack2(a.q_scale, a.q_scale);
+  #pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+          const int t4 = half * 16 + tg * 4;
+          uint64_t run01 = half == 0 ? pack2(run0[0][0], run0[0][1]) : pack2(run0[1][0], run0[1][1]);
+          uint64_t run23 = half == 0 ? pack2(run0[0][2], run0[0][3]) : pack2(run0[1][2], run0[1][3]);
+          const uint64_t ref01 = half == 0 ? pack2(refL[0], refL[1]) : 0ull, ref23 = half == 0 ? pack2(refL[2], refL[3]) : 0ull;
+  #pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int t = t4 + j;
+            const uint32_t off_k = OFF_KQ + sw128_offset(64, t, c0), off_q = OFF_KQ + sw128_offset(64, 32 + t, c0);
+            const uint32_t off_h = OFF_KH + sw128_offset(32, t, c0);
+            const uint2 kw = *reinterpret_cast<const uint2 *>(smem + off_k);
             const float4 g4 = *reinterpret_cast<const float4 *>(smem + off_h);
-            g01 = pack2(g4.x, g4.y);
-            g23 = pack2(g4.z, g4.w);
-          } else {
-            const float gs = gsc_s[(ch & 3) * C + t];
-            g01 = g23 = pack2(gs, gs);
+            const uint64_t g01 = pack2(g4.x, g4.y), g23 = pack2(g4.z, g4.w);
+            const uint64_t k01 = pack2(bf16lo(kw.x), bf16hi(kw.x)), k23 = pack2(bf16lo(kw.y), bf16hi(kw.y));
+            run01 = add2(run01, g01);
+            run23 = add2(run23, g23);
+            const uint64_t d01 = fma2(run01, l2e2, ref01), d23 = fma2(run23, l2e2, ref23);  // (G_t - G_m) log2(e)
+            float d[4], dc[4];
+            unpack2(d01, d[0], d[1]);
+            unpack2(d23, d[2], d[3]);
+            unpack2(add2(d01, comp2), dc[0], dc[1]);
+            unpack2(add2(d23, comp2), dc[2], dc[3]);
+            const uint64_t e1_01 = pack2(ex2f(dc[0]), ex2f(dc[1])), e1_23 = pack2(ex2f(dc[2]), ex2f(dc[3]));
+            const uint64_t e2_01 = pack2(ex2f(-d[0]), ex2f(-d[1])), e2_23 = pack2(ex2f(-d[2]), ex2f(-d[3]));
+            float kt[4], kh[4];
+            unpack2(mul2(k01, e1_01), kt[0], kt[1]);
+            unpack2(mul2(k23, e1_23), kt[2], kt[3]);
+            unpack2(mul2(k01, e2_01), kh[0], kh[1]);
+            unpack2(mul2(k23, e2_23), kh[2], kh[3]);
+            if (WITH_O) {
+              const uint2 qw = *reinterpret_cast<const uint2 *>(smem + off_q);
+              const uint64_t q01 = pack2(bf16lo(qw.x), bf16hi(qw.x)), q23 = pack2(bf16lo(qw.y), bf16hi(qw.y));
+              float qt[4];
+              unpack2(mul2(q01, mul2(e1_01, qs2)), qt[0], qt[1]);
+              unpack2(mul2(q23, mul2(e1_23, qs2)), qt[2], qt[3]);
+              *reinterpret_cast<uint4 *>(smem + off_q) =
+                  make_uint4(tf32_pre(qt[0]), tf32_pre(qt[1]), tf32_pre(qt[2]), tf32_pre(qt[3]));
+            }
+            *reinterpret_cast<uint4 *>(smem + off_k) =
+                make_uint4(tf32_pre(kt[0]), tf32_pre(kt[1]), tf32_pre(kt[2]), tf32_pre(kt[3]));
+            // Kh goes out twice, the same four values in both places: K-major (MMA1 contracts over the channels) and
+            // MN-major (MMA5 contracts over the tokens).  A tf32 MN-major operand has a swizzle of its own, so the two
+            // tiles differ in where a vector lands, not in what it holds.
+            const uint4 khv = make_uint4(tf32_pre(kh[0]), tf32_pre(kh[1]), tf32_pre(kh[2]), tf32_pre(kh[3]));
+            *reinterpret_cast<uint4 *>(smem + off_h) = khv;
+            *reinterpret_cast<uint4 *>(kht_tile + mn32_offset(32, t, c0)) = khv;
           }
-          const uint64_t k01 = pack2(bf16lo(kw.x), bf16hi(kw.x)), k23 = pack2(bf16lo(kw.y), bf16hi(kw.y));
-          run01 = add2(run01, g01);
-          run23 = add2(run23, g23);
-          const uint64_t d01 = fma2(run01, l2e2, ref01), d23 = fma2(run23, l2e2, ref23);  // (G_t - G_m) log2(e)
-          float d[4], dc[4];
-          unpack2(d01, d[0], d[1]);
-          unpack2(d23, d[2], d[3]);
-          unpack2(add2(d01, comp2), dc[0], dc[1]);
-          unpack2(add2(d23, comp2), dc[2], dc[3]);
-          const uint64_t e1_01 = pack2(ex2f(dc[0]), ex2f(dc[1])), e1_23 = pack2(ex2f(dc[2]), ex2f(dc[3]));
-          const uint64_t e2_01 = pack2(ex2f(-d[0]), ex2f(-d[1])), e2_23 = pack2(ex2f(-d[2]), ex2f(-d[3]));
-          float kt[4], kh[4];
-          unpack2(mul2(k01, e1_01), kt[0], kt[1]);
-          unpack2(mul2(k23, e1_23), kt[2], kt[3]);
-          unpack2(mul2(k01, e2_01), kh[0], kh[1]);
-          unpack2(mul2(k23, e2_23), kh[2], kh[3]);
-          if (WITH_O) {
-            const uint2 qw = *reinterpret_cast<const uint2 *>(smem + off_q);
-            const uint64_t q01 = pack2(bf16lo(qw.x), bf16hi(qw.x)), q23 = pack2(bf16lo(qw.y), bf16hi(qw.y));
-            float qt[4];
-            unpack2(mul2(q01, mul2(e1_01, qs2)), qt[0], qt[1]);
-            unpack2(mul2(q23, mul2(e1_23, qs2)), qt[2], qt[3]);
-            *reinterpret_cast<uint4 *>(smem + off_q) =
-                make_uint4(tf32_pre(qt[0]), tf32_pre(qt[1]), tf32_pre(qt[2]), tf32_pre(qt[3]));
-          }
-          *reinterpret_cast<uint4 *>(smem + off_k) =
-              make_uint4(tf32_pre(kt[0]), tf32_pre(kt[1]), tf32_pre(kt[2]), tf32_pre(kt[3]));
-          // Kh goes out twice, the same four values in both places: K-major (MMA1 contracts over the channels) and
-          // MN-major (MMA5 contracts over the tokens).  A tf32 MN-major operand has a swizzle of its own, so the two
-          // tiles differ in where a vector lands, not in what it holds.
-          const uint4 khv = make_uint4(tf32_pre(kh[0]), tf32_pre(kh[1]), tf32_pre(kh[2]), tf32_pre(kh[3]));
-          *reinterpret_cast<uint4 *>(smem + off_h) = khv;
-          *reinterpret_cast<uint4 *>(kht_tile + mn32_offset(32, t, c0)) = khv;
         }
+        // the exponents of this chunk may have overflowed: the unit will not be written back.  (Every lane of a channel
+        // quad holds the same totals; having only the first token group store keeps the producer loop free of spills.)
+        if (out_of_range && tg == 0) misc->domain_flag = 1;
+      } else {
+        // ---- GDN: one scalar log-decay per token.  The first producer warp (lane = token) forms the running sums and
+        // the per-token factors; nothing per channel needs an exponential, and k, q stay exactly their bf16 values:
+        //   e1_t = exp(G_t - G_m), e2_t = exp(G_m - G_t) with m the end of the first half;
+        //   MMA1 works on raw k, q (bf16 tile), MMA2 on raw k, q widened to tf32 containers, MMA5 on k_t e2_t;
+        //   e1_t goes onto the rows of A, R and the outputs where they leave tensor memory, e2_j onto the columns of A, P.
+        bool out_of_range = false;
+        if (ptid < C) {
+          const int slot = (ch & 3) * C + lane;
+          float incl = gsc_cur;
+#pragma unroll
+          for (int dlt = 1; dlt < 32; dlt <<= 1) {
+            const float x = __shfl_up_sync(0xffffffffu, incl, dlt);
+            if (lane >= dlt) incl += x;
+          }
+          const float tot0 = __shfl_sync(0xffffffffu, incl, 15);          // G_m: the first half's total
+          const float tot1 = __shfl_sync(0xffffffffu, incl, 31) - tot0;   // G_C - G_m
+          const float d2 = (incl - tot0) * LOG2E;
+          const float e1 = ex2f(d2), e2 = ex2f(-d2);
+          e1c_s[slot] = e1 * kTruncComp;
+          e2_s[slot] = e2;
+          bte1_s[slot] = beta_s[slot] * e1;
+          out_of_range = !(fabsf(tot0) <= kMaxHalfDecay) || !(fabsf(tot1) <= kMaxHalfDecay);   // also true for NaN
+          // state factor from where the previous chunk left the state to this chunk's midpoint, and the factor owed after
+          // it; scalars here, written for every channel so that the chain warps read them as they do for KDA
+          const float f = ex2f((post_prev + tot0) * LOG2E);
+          post_prev = tot1;
+          *reinterpret_cast<float4 *>(fac_s + par * D + lane * 4) = make_float4(f, f, f, f);
+          *reinterpret_cast<float4 *>(post_s + par * D + lane * 4) = make_float4(tot1, tot1, tot1, tot1);
+        }
+        mbar_arrive(&misc->rdy_fac[par]);
+        asm volatile("bar.sync 2, 128;" ::: "memory");   // the factors are visible to all producer warps
+        asm volatile("cp.async.wait_group 0;" ::: "memory");  // k and q have landed
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int t = half * 16 + tg * 4 + j;
+            const uint32_t off_k = OFF_KQ + sw128_offset(64, t, c0), off_q = OFF_KQ + sw128_offset(64, 32 + t, c0);
+            const uint2 kw = *reinterpret_cast<const uint2 *>(smem + off_k);
+            const uint4 kf = make_uint4(kw.x << 16, kw.x & 0xFFFF0000u, kw.y << 16, kw.y & 0xFFFF0000u);  // exact
+            *reinterpret_cast<uint4 *>(smem + off_k) = kf;
+            *reinterpret_cast<uint2 *>(smem + OFF_KQ16 + sw128_offset_bf16(64, t, c0)) = kw;
+            if (WITH_O) {
+              const uint2 qw = *reinterpret_cast<const uint2 *>(smem + off_q);
+              *reinterpret_cast<uint4 *>(smem + off_q) = make_uint4(qw.x << 16, qw.x & 0xFFFF0000u, qw.y << 16, qw.y & 0xFFFF0000u);
+              *reinterpret_cast<uint2 *>(smem + OFF_KQ16 + sw128_offset_bf16(64, 32 + t, c0)) = qw;
+            }
+            const float e2 = e2_s[(ch & 3) * C + t];
+            *reinterpret_cast<uint4 *>(kht_tile + mn32_offset(32, t, c0)) =
+                make_uint4(tf32_pre(__uint_as_float(kf.x) * e2), tf32_pre(__uint_as_float(kf.y) * e2),
+                           tf32_pre(__uint_as_float(kf.z) * e2), tf32_pre(__uint_as_float(kf.w) * e2));
+          }
+        }
+        if (out_of_range && lane == 0) misc->domain_flag = 1;
       }
-      // the exponents of this chunk may have overflowed: the unit will not be written back.  (Every lane of a channel
-      // quad holds the same totals; having only the first token group store keeps the producer loop free of spills.)
-      if (out_of_range && tg == 0) misc->domain_flag = 1;
       fence_smem_to_async();
       mbar_arrive(&misc->rdy_prep);  // -> MMA1
     }
@@ -722,13 +787,19 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         tmem_ld_wait();
         const int t = lane;
         // row t of P = lower_incl_diag(Qt Kh^T), straight to its operand tile
+        // (GDN: the raw q_t . k_j gets its column factor e2_j here; the row factor e1_t is applied to the outputs)
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
+          float4 e2 = make_float4(kInvTruncComp, kInvTruncComp, kInvTruncComp, kInvTruncComp);
+          if constexpr (!KDA) {
+            e2 = *reinterpret_cast<const float4 *>(e2_s + (ch & 3) * C + j);
+            e2.x *= kInvTruncComp; e2.y *= kInvTruncComp; e2.z *= kInvTruncComp; e2.w *= kInvTruncComp;
+          }
           uint4 o;
-          o.x = (j + 0 <= t) ? tf32_pre(__uint_as_float(x[j + 0]) * kInvTruncComp) : 0u;
-          o.y = (j + 1 <= t) ? tf32_pre(__uint_as_float(x[j + 1]) * kInvTruncComp) : 0u;
-          o.z = (j + 2 <= t) ? tf32_pre(__uint_as_float(x[j + 2]) * kInvTruncComp) : 0u;
-          o.w = (j + 3 <= t) ? tf32_pre(__uint_as_float(x[j + 3]) * kInvTruncComp) : 0u;
+          o.x = (j + 0 <= t) ? tf32_pre(__uint_as_float(x[j + 0]) * e2.x) : 0u;
+          o.y = (j + 1 <= t) ? tf32_pre(__uint_as_float(x[j + 1]) * e2.y) : 0u;
+          o.z = (j + 2 <= t) ? tf32_pre(__uint_as_float(x[j + 2]) * e2.z) : 0u;
+          o.w = (j + 3 <= t) ? tf32_pre(__uint_as_float(x[j + 3]) * e2.w) : 0u;
           *reinterpret_cast<uint4 *>(smem + OFF_PM + sw128_offset(32, t, j)) = o;
         }
         fence_smem_to_async();
@@ -748,7 +819,9 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           const float vv = __bfloat162float(Vs[(tb + j) * D + vrow]);
-          const float rhs = beta_c[tb + j] * (vv - __uint_as_float(x[j]));
+          // GDN: the product is k_t S' on the raw keys; its row factor e1_t (with the truncation compensation) comes here
+          const float r = KDA ? __uint_as_float(x[j]) : e1c_s[(ch & 3) * C + tb + j] * __uint_as_float(x[j]);
+          const float rhs = beta_c[tb + j] * (vv - r);
           x[j] = to_tf32(rhs);
           lo[j] = tf32_pre(rhs - __uint_as_float(x[j]));
         }
@@ -787,6 +860,13 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         uint32_t x[16];
         tmem_ld16(tlane + COL_RO + 32 + tb, x);
         tmem_ld_wait();
+        if constexpr (!KDA) {
+          // GDN: the accumulated q_t (S' + sum_j e2_j k_j u_j^T) still lacks its row factor e1_t, the query scale and
+          // the truncation compensation
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            x[j] = __float_as_uint(__uint_as_float(x[j]) * (e1c_s[(ch & 3) * C + tb + j] * a.q_scale));
+        }
         if constexpr (sizeof(OT) == 2) {
           // through shared memory (the T and P tiles are free now) so that global stores are 16 bytes wide
           __nv_bfloat16 *Os = reinterpret_cast<__nv_bfloat16 *>(smem + OFF_TM);

@@ -156,6 +156,13 @@ __device__ __forceinline__ uint32_t sw128_offset(uint32_t rows, uint32_t r, uint
   return blk * rows * 128u + r * 128u + ((((cin >> 2) ^ (r & 7u)) << 4) | ((cin & 3u) << 2));
 }
 
+// The same canonical K-major layout for 16-bit elements: 64 columns per 128-byte row.  `col` must be a multiple of 4
+// (8 bytes) for the 8-byte accesses made here.
+__device__ __forceinline__ uint32_t sw128_offset_bf16(uint32_t rows, uint32_t r, uint32_t col) {
+  const uint32_t blk = col >> 6, cin = col & 63;
+  return blk * rows * 128u + r * 128u + ((((cin >> 3) ^ (r & 7u)) << 4) | ((cin & 7u) << 1));
+}
+
 // MN-major tf32 operand tiles (rows = K index, the M or N index contiguous along a row): the tensor core accepts one
 // swizzle for them, the 128-byte swizzle on 32-byte units.  A tile of R rows (the K index) and 32*NB tf32 columns is
 // stored as NB blocks of [R rows][128 bytes]; inside a block the 32-byte unit u of row r sits at unit position
@@ -182,6 +189,20 @@ __device__ __forceinline__ uint64_t desc_mn32(uint32_t smem_addr, uint32_t block
 __host__ __device__ constexpr uint32_t idesc_tf32(uint32_t M, uint32_t N, bool a_mn_major, bool b_mn_major) {
   return (1u << 4) | (2u << 7) | (2u << 10) | (uint32_t(a_mn_major) << 15) | (uint32_t(b_mn_major) << 16) |
          ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+// Instruction descriptor, kind::f16 with bf16 operands (both K-major), fp32 accumulation.
+__host__ __device__ constexpr uint32_t idesc_bf16(uint32_t M, uint32_t N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] * B[smem], bf16 operands; one K = 16 slice.
+__device__ __forceinline__ void mma_ss_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(uint32_t(accumulate))
+      : "memory");
 }
 
 // D[tmem] (+)= A[smem] * B[smem]; one K = 8 slice.  Issued by a single thread.
