@@ -43,12 +43,19 @@ TF32_OVER_BF16 = 0.489        # nominal dense 1.1 : 2.25
 CHUNKED_FLOPS_PER_TOKEN_HEAD = 196608   # tf32 flops the chunked kernel issues per (token, head): 32-token chunks,
                                         # MMA1 padded to M = 128, hi/lo pairs in MMA3, MMA4 and MMA5
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes, from one ncu full-set capture of
-# the KDA serving workload at 8 requests and a 128-token suffix (a full-size launch is too large to capture); every
-# request and token moves the same bytes, so traffic grows in proportion and a full launch is scaled by its units.
-# Below 1.0 = lines still dirty in L2 when the kernel ended, not skipped work.
-NCU_TRAFFIC_OVER_ALGORITHMIC = {"pack": 255.99e6 / 306.12e6, "restore": 500.13e6 / 555.71e6,
-                                "refresh_chunked": 1.9830e9 / 2.0164e9}
+# Traffic of a launch over its algorithmic bytes, from one ncu capture of the KDA serving workload at 8 requests and a
+# 128-token suffix (a full-size launch is too large to capture; every request and token moves the same bytes, so traffic
+# grows in proportion and a full launch is scaled by its units).  Traffic = dram__bytes_read.sum + 32 B x
+# lts__t_sectors_srcunit_tex_op_write.sum (the sectors the SMs wrote into L2): the DRAM write counter alone misses the
+# lines still dirty in the 126 MB L2 when the kernel ends (a third of the pack's writes at this size), and
+# lts__t_sectors_op_write.sum counts a sector once more when its home L2 slice is on the other die (1.5000x the
+# algorithmic write bytes for all three kernels).  profiles/traffic_kda_serving.md has the numbers.
+NCU_CAPTURE = {  # kernel: (dram__bytes_read.sum, lts__t_sectors_srcunit_tex_op_write.sum, algorithmic bytes of that launch)
+    "pack": (153370624, 4783104, 306118656),
+    "restore": (153463296, 12582912, 555712512),
+    "refresh_chunked": (1412594688, 18874368, 2016411648),
+}
+NCU_TRAFFIC_OVER_ALGORITHMIC = {k: (rd + 32 * wr) / alg for k, (rd, wr, alg) in NCU_CAPTURE.items()}
 
 CONFIGS = {
     1: dict(name="kda_serving", kind="KDA", L=24, H_v=32, H_k=32, n_req=64, keep=0.38, rate_lo=1e-3, suffix=256, seed=1),
@@ -292,6 +299,7 @@ def main():
                     help="checkpoint pool format: fp32 bit copies, or the Appendix D INT8 codec fused into pack/restore")
     ap.add_argument("--pool-slots", type=int, default=2048, help="config 4: slots of the bounded checkpoint pool")
     ap.add_argument("--trace-rounds", type=int, default=0, help="config 4: replay only the first rounds of the trace")
+    ap.add_argument("--tp-ranks", type=int, default=8, help="virtual TP ranks of the placement leg (0 or 1 = skip it)")
     ap.add_argument("--dry-launch", action="store_true", help="start the ranks, count them over gloo, do no GPU work")
     args = ap.parse_args()
     world_env = int(os.environ.get("WORLD_SIZE", "1"))
@@ -453,6 +461,38 @@ def main():
     assert dasc.dasc_refresh_status(ws) == 0
     (t_window,) = max_over_ranks([ev_w[0].elapsed_time(ev_w[1]) / args.steps], dev)
 
+    # ---- Section 4.3 on the device: the same Store / Load with TP-balanced placement, timed apart from the step.
+    #      Eight virtual ranks (eight pool buffers on this GPU, as peer mappings would appear to one rank); this rank
+    #      holds the heaviest payload, so most of its units are pushed into the other ranks' pools. ----
+    tp = None
+    if args.layout == "ragged" and not int8 and args.tp_ranks > 1:
+        Tn = args.tp_ranks
+        U = np.full(Tn, int(plan.units_retained) // 4, np.int64)
+        U[0] = int(plan.units_retained)
+        width, _ = dasc.dasc_tp_balance(U)
+        tp_pools = [torch.empty((N_REQ, width * int(plan.unit_floats)), device=dev) for _ in range(Tn)]
+        for _ in range(3):
+            dasc.dasc_pack_tp(plan, state, layer_stride, req_stride, ids, tp_pools, U, 0, slots)
+            dasc.dasc_restore_tp(plan, tp_pools, U, 0, slots, active, layer_stride, req_stride, ids)
+        barrier()
+        ev_t = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        n_it = 5
+        ev_t[0].record(stream)
+        for _ in range(n_it):
+            dasc.dasc_pack_tp(plan, state, layer_stride, req_stride, ids, tp_pools, U, 0, slots)
+        ev_t[1].record(stream)
+        for _ in range(n_it):
+            dasc.dasc_restore_tp(plan, tp_pools, U, 0, slots, active, layer_stride, req_stride, ids)
+        ev_t[2].record(stream)
+        barrier()
+        t_ptp, t_rtp = max_over_ranks([ev_t[0].elapsed_time(ev_t[1]) / n_it, ev_t[1].elapsed_time(ev_t[2]) / n_it], dev)
+        tp = {"virtual_ranks": Tn, "units_per_rank": U.tolist(), "slot_width_units": width,
+              "pack_tp_GBps": pack_bytes / (t_ptp * 1e-3) / 1e9, "restore_tp_GBps": restore_bytes / (t_rtp * 1e-3) / 1e9,
+              "ms_pack_tp": t_ptp, "ms_restore_tp": t_rtp,
+              "note": "all pools local to this GPU (one GPU in this run): the figures show the cost of the placement "
+                      "arithmetic, not of NVLink"}
+        del tp_pools
+
     # ---- end-to-end leg: host buffers, copies inside the timed region -------------------------
     e2e = None
     if not args.no_e2e:
@@ -603,6 +643,8 @@ def main():
         # the units handed to it (AUTO); a single refresh kernel per group when an algorithm is forced
         "gpu_launches": (2 + n_groups * (2 if args.algo == "auto" else 1)) * args.steps,
     }
+    if tp:
+        line["tp_placement"] = tp
     if e2e:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1 and not args.mixed_heads:  # the oracle leg times the per-layer rule

@@ -337,8 +337,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         mma_commit(&misc->bar_ap);
       }
       __syncwarp();
-      // MMA2: S'^T [Kt;Qt]^T, the fp32 state read as a tf32 operand.  The state pass hands the channels over in two
-      // halves (each chain warp scales 32 of its 64 columns at a time): slices 0-3 and 8-11 first, then 4-7 and 12-15.
+      // MMA2: S'^T [Kt;Qt]^T, the fp32 state read as a tf32 operand
       if (lane == 0) wait_bar(&misc->rdy_state, par, misc, err);
       __syncwarp();
       if (lane == 0) {
