@@ -928,6 +928,23 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   if (warp == WARP_MMA) tmem_dealloc(tm, TMEM_COLS);
 }
 
+// cuTensorMapEncodeTiled is a driver entry point.  It is looked up through the runtime at first use, so that the library
+// has no link-time dependency on libcuda and still loads (plan building, accessors) on a machine without a driver.
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
 template <bool KDA, typename OT, bool WITH_O>
 int launch(const DascRefreshArgs &a, void *stream) {
   auto kern = refresh_chunked_kernel<KDA, OT, WITH_O>;
@@ -947,7 +964,9 @@ int launch(const DascRefreshArgs &a, void *stream) {
     const cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * 4, static_cast<cuuint64_t>(a.H_v) * D * 4};
     const cuuint32_t box[3] = {32, 1, static_cast<cuuint32_t>(C)};
     const cuuint32_t ones[3] = {1, 1, 1};
-    if (cuTensorMapEncodeTiled(&tmap_g, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.g), dims, strides, box, ones,
+    const EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return static_cast<int>(cudaErrorNotSupported);
+    if (encode(&tmap_g, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.g), dims, strides, box, ones,
                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return static_cast<int>(cudaErrorInvalidValue);
