@@ -65,7 +65,7 @@ def test_gdn_headwise_config_pack_restore_refresh():
     dasc.dasc_refresh(plan, active, ls, rs, ids, q, k, v, g, beta, cu.to(dev), T, suffix, o=o, workspace=ws)
     torch.cuda.synchronize()
     assert dasc.dasc_refresh_status(ws) == 0
-    units = sample_units(2, n_req, L, H_v, 24)
+    units = sample_units(2, n_req, L, H_v, 96)
     worst = check_sampled_refresh(dasc.GDN, plan, oplan, before, active, ls, rs, q, k, v, g, beta, o, cu, units, TOL)
     print("GDN config: worst sampled rel err", worst)
 
@@ -104,7 +104,7 @@ def test_aggressive_kda_refresh_config(suffix):
                           layer_end=lb + group, o=o, workspace=ws)
         torch.cuda.synchronize()
         assert dasc.dasc_refresh_status(ws) == 0
-        units = sample_units(suffix + lb, n_req, group, H, 6 if suffix == 4096 else 12)
+        units = sample_units(suffix + lb, n_req, group, H, 8 if suffix == 4096 else 32)
         worst = max(worst, check_sampled_refresh(dasc.KDA, plan, oplan, before, active, ls, rs, q, k, v, g, beta, o,
                                                  cu, units, TOL, layer_begin=lb))
         # layers outside the group are untouched
@@ -215,7 +215,7 @@ def test_kda_serving_config_refresh_in_the_benchmarks_launch():
     dasc.dasc_refresh(plan, active, ls, rs, ids, q, k, v, g, beta, cu.to(dev), T, suffix, o=o, workspace=ws)
     torch.cuda.synchronize()
     assert dasc.dasc_refresh_status(ws) == 0
-    units = sample_units(11, n_req, L, H, 16)
+    units = sample_units(11, n_req, L, H, 128)
     # bf16 outputs carry their own rounding (half an ulp is up to 2^-8 of the value): states at 1e-3, outputs at 1e-3 + 2^-8
     worst = check_sampled_refresh(dasc.KDA, plan, oplan, before, active, ls, rs, q, k, v, g, beta, None, cu, units, TOL)
     worst_o = check_sampled_refresh(dasc.KDA, plan, oplan, before, active, ls, rs, q, k, v, g, beta, o, cu, units,
