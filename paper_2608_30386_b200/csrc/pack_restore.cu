@@ -28,6 +28,9 @@ struct TpPools {
   uint32_t unit_begin;             // global position of this rank's first packed unit
   uint32_t width;                  // C: units per rank and slot
   uint32_t unit_vecs;              // 16-byte vectors per unit
+  int32_t unit_shift;              // log2(unit_vecs) when that is a power of two, else -1
+  uint32_t width_magic;            // owner = umulhi(pos, width_magic) >> width_shift for every pos < 2^31 (width >= 2)
+  uint32_t width_shift;
 };
 
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
@@ -47,10 +50,11 @@ __device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v) {
 // Where vector `pv` (counted over the whole packed slot of this rank) of slot `slot` lives under the TP-balanced
 // placement.
 __device__ __forceinline__ uint4 *tp_address(const TpPools &tp, int64_t slot, int64_t slot_stride4, uint32_t pv) {
-  const uint32_t unit = pv / tp.unit_vecs;
+  // both divisions by multiplication or shift: they sit in front of every 16-byte access
+  const uint32_t unit = tp.unit_shift >= 0 ? pv >> tp.unit_shift : pv / tp.unit_vecs;
   const uint32_t in_unit = pv - unit * tp.unit_vecs;
   const uint32_t pos = tp.unit_begin + unit;
-  const uint32_t owner = pos / tp.width;
+  const uint32_t owner = tp.width > 1 ? __umulhi(pos, tp.width_magic) >> tp.width_shift : pos;
   const uint32_t local = pos - owner * tp.width;
   return tp.base[owner] + slot * slot_stride4 + static_cast<int64_t>(local) * tp.unit_vecs + in_unit;
 }
@@ -181,6 +185,17 @@ TpPools make_tp(const DascTpPlacement *p, int64_t unit_floats) {
     tp.unit_begin = static_cast<uint32_t>(p->unit_begin);
     tp.width = static_cast<uint32_t>(p->width);
     tp.unit_vecs = static_cast<uint32_t>(unit_floats / 4);
+    tp.unit_shift = -1;
+    for (int sft = 0; sft < 31; ++sft)
+      if ((1u << sft) == tp.unit_vecs) tp.unit_shift = sft;
+    if (tp.width > 1) {
+      // division of a 31-bit number by `width`: with s = ceil(log2 width), m = floor(2^(31+s) / width) + 1 < 2^32 and
+      // floor(pos / width) = (pos * m) >> (31 + s) for every pos < 2^31
+      uint32_t sft = 0;
+      while ((uint64_t{1} << sft) < tp.width) ++sft;
+      tp.width_magic = static_cast<uint32_t>((uint64_t{1} << (31 + sft)) / tp.width + 1);
+      tp.width_shift = sft - 1;
+    }
   }
   return tp;
 }
