@@ -49,7 +49,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
   return false;
 }
 
-// ---- TMA (bulk tensor copies into shared memory, completing on an mbarrier; never with cluster multicast) ----
+// ---- TMA (bulk tensor copies into this CTA's shared memory, completing on an mbarrier; one CTA, one destination) ----
 // The issuing thread announces the bytes of the copy it is about to start (this is also its arrival).
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
