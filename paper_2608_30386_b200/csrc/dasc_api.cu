@@ -1,6 +1,7 @@
 // C ABI of libdasc: argument validation and marshalling only; all work happens
 // in plan_host.cpp (host plan) and in the CUDA kernels.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cstring>
@@ -11,6 +12,15 @@
 namespace {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// A named range around each device call of the ABI, visible in a timeline when a profiler is attached (header-only
+// NVTX: without a tool the calls do nothing).
+struct TraceRange {
+  explicit TraceRange(const char *name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange &) = delete;
+  TraceRange &operator=(const TraceRange &) = delete;
+};
 
 struct DeviceGuard {
   int prev = -1;
@@ -168,6 +178,7 @@ dasc_status_t dasc_plan_layer_offsets(const dasc_plan_t *plan, int64_t *out) { D
 dasc_status_t dasc_pack(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride, int64_t req_stride,
                         const int32_t *src_req, float *pool_base, int64_t slot_stride, const int32_t *dst_slot,
                         int32_t n_pairs, void *cuda_stream) {
+  TraceRange trace("dasc_pack");
   dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, src_req, pool_base, &slot_stride,
                                      dst_slot, n_pairs);
   if (st != DASC_OK || n_pairs == 0) return st;
@@ -179,6 +190,7 @@ dasc_status_t dasc_pack(const dasc_plan_t *plan, const float *state_base, int64_
 dasc_status_t dasc_restore(const dasc_plan_t *plan, const float *pool_base, int64_t slot_stride,
                            const int32_t *src_slot, float *state_base, int64_t layer_stride, int64_t req_stride,
                            const int32_t *dst_req, int32_t n_pairs, void *cuda_stream) {
+  TraceRange trace("dasc_restore");
   dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, dst_req, pool_base, &slot_stride,
                                      src_slot, n_pairs);
   if (st != DASC_OK || n_pairs == 0) return st;
@@ -196,6 +208,7 @@ dasc_status_t dasc_padded_pool_floats(const dasc_plan_t *plan, int64_t n_slots, 
 dasc_status_t dasc_pack_padded(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride,
                                int64_t req_stride, const int32_t *src_req, float *pool_base, int64_t n_slots,
                                const int32_t *dst_slot, int32_t n_pairs, void *cuda_stream) {
+  TraceRange trace("dasc_pack_padded");
   int64_t unused = 0;
   dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, src_req, pool_base, &unused, dst_slot,
                                      n_pairs);
@@ -209,6 +222,7 @@ dasc_status_t dasc_pack_padded(const dasc_plan_t *plan, const float *state_base,
 dasc_status_t dasc_restore_padded(const dasc_plan_t *plan, const float *pool_base, int64_t n_slots,
                                   const int32_t *src_slot, float *state_base, int64_t layer_stride,
                                   int64_t req_stride, const int32_t *dst_req, int32_t n_pairs, void *cuda_stream) {
+  TraceRange trace("dasc_restore_padded");
   int64_t unused = 0;
   dasc_status_t st = check_copy_args(plan, state_base, layer_stride, req_stride, dst_req, pool_base, &unused, src_slot,
                                      n_pairs);
@@ -340,6 +354,7 @@ dasc_status_t dasc_pack_tp(const dasc_plan_t *plan, const float *state_base, int
                            const int32_t *src_req, float *const *pool_bases, const int64_t *units_per_rank,
                            int32_t n_ranks, int32_t rank, int64_t slot_stride, const int32_t *dst_slot,
                            int32_t n_pairs, void *cuda_stream) {
+  TraceRange trace("dasc_pack_tp");
   DascTpPlacement pl{};
   dasc_status_t st = check_tp_args(plan, pool_bases, units_per_rank, n_ranks, rank, &slot_stride, &pl);
   if (st != DASC_OK) return st;
@@ -355,6 +370,7 @@ dasc_status_t dasc_restore_tp(const dasc_plan_t *plan, float *const *pool_bases,
                               int32_t n_ranks, int32_t rank, int64_t slot_stride, const int32_t *src_slot,
                               float *state_base, int64_t layer_stride, int64_t req_stride, const int32_t *dst_req,
                               int32_t n_pairs, void *cuda_stream) {
+  TraceRange trace("dasc_restore_tp");
   DascTpPlacement pl{};
   dasc_status_t st = check_tp_args(plan, pool_bases, units_per_rank, n_ranks, rank, &slot_stride, &pl);
   if (st != DASC_OK) return st;
@@ -419,6 +435,7 @@ dasc_status_t dasc_int8_slot_bytes(const dasc_plan_t *plan, size_t *out) {
 dasc_status_t dasc_pack_int8(const dasc_plan_t *plan, const float *state_base, int64_t layer_stride,
                              int64_t req_stride, const int32_t *src_req, void *pool_base, int64_t slot_stride_bytes,
                              const int32_t *dst_slot, int32_t n_pairs, void *cuda_stream) {
+  TraceRange trace("dasc_pack_int8");
   dasc_status_t st = check_int8_args(plan, state_base, layer_stride, req_stride, src_req, pool_base,
                                      &slot_stride_bytes, dst_slot, n_pairs);
   if (st != DASC_OK || n_pairs == 0) return st;
@@ -430,6 +447,7 @@ dasc_status_t dasc_pack_int8(const dasc_plan_t *plan, const float *state_base, i
 dasc_status_t dasc_restore_int8(const dasc_plan_t *plan, const void *pool_base, int64_t slot_stride_bytes,
                                 const int32_t *src_slot, float *state_base, int64_t layer_stride, int64_t req_stride,
                                 const int32_t *dst_req, int32_t n_pairs, void *cuda_stream) {
+  TraceRange trace("dasc_restore_int8");
   dasc_status_t st = check_int8_args(plan, state_base, layer_stride, req_stride, dst_req, pool_base,
                                      &slot_stride_bytes, src_slot, n_pairs);
   if (st != DASC_OK || n_pairs == 0) return st;
@@ -569,6 +587,7 @@ dasc_status_t dasc_refresh(const dasc_plan_t *plan, float *state_base, int64_t l
                            int64_t total_tokens, int32_t max_seqlen, int32_t layer_begin, int32_t layer_end,
                            float q_scale, void *o, int32_t o_dtype, int32_t mode, int32_t algo, void *workspace,
                            size_t workspace_bytes, void *cuda_stream) {
+  TraceRange trace("dasc_refresh");
   if (!q) return n_req == 0 || total_tokens == 0 || layer_end == layer_begin ? DASC_OK : DASC_ERR_INVALID_ARG;
   RefreshRequest rq;
   const dasc_status_t st = refresh_validate(plan, state_base, layer_stride, req_stride, req_idx, q, k, v, io_dtype, g,
@@ -585,6 +604,7 @@ dasc_status_t dasc_refresh_window(const dasc_plan_t *plan, float *state_base, in
                                   int32_t layer_begin, int32_t layer_end, float q_scale, void *o, int32_t o_dtype,
                                   int32_t algo, int32_t *window_begin, void *workspace, size_t workspace_bytes,
                                   void *cuda_stream) {
+  TraceRange trace("dasc_refresh_window");
   if (!plan || plan->info.device < 0 || n_req < 0) return DASC_ERR_INVALID_ARG;
   if (o && !q) return DASC_ERR_INVALID_ARG;
   if (window <= 0) window = plan->info.w_replay;
