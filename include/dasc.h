@@ -148,6 +148,18 @@ typedef struct {
 dasc_status_t dasc_plan(const dasc_plan_desc_t *desc, int32_t device, dasc_plan_t **out);
 void dasc_plan_destroy(dasc_plan_t *plan);
 
+/*
+ * A plan depends on model weights only (Section 4.1: built once offline), so it can be built where the weights are
+ * and shipped to the serving processes.  dasc_plan_save writes a self-contained little-endian blob of
+ * dasc_plan_save_bytes() bytes into the HOST buffer `buf` (scores, mask, windows and the scalar results; the index
+ * tables are derived again on load); dasc_plan_load checks the blob (magic, version, sizes, that the counts it claims
+ * are those of its mask) and rebuilds the plan, uploading its tables to `device` as dasc_plan does (device < 0: host
+ * only).  A blob that fails a check gives DASC_ERR_INVALID_ARG and *out = NULL.
+ */
+dasc_status_t dasc_plan_save_bytes(const dasc_plan_t *plan, size_t *out);
+dasc_status_t dasc_plan_save(const dasc_plan_t *plan, void *buf, size_t buf_bytes);
+dasc_status_t dasc_plan_load(const void *buf, size_t bytes, int32_t device, dasc_plan_t **out);
+
 /* Accessors.  Array outputs are HOST buffers the caller sized from dasc_plan_info:
  * horizon/mask/window: n_layers*units_per_layer entries, [layer][unit];
  * layer_counts: n_layers (r_l); layer_offsets: n_layers+1 (o_l). */

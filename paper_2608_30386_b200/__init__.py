@@ -11,5 +11,5 @@ from .binding import (  # noqa: F401
     dasc_int8_slot_bytes, dasc_pack_int8, dasc_restore, dasc_restore_int8, lib, status_string, version,
     LAYOUT_DENSE, LAYOUT_PADDED, LAYOUT_RAGGED, dasc_checkpoint_bytes, dasc_pack_padded, dasc_padded_pool_floats,
     dasc_restore_padded, dasc_slot_budget, dasc_tp_balance, dasc_pack_tp, dasc_restore_tp, dasc_tp_head_permutation,
-    dasc_conv_store, dasc_conv_load, dasc_refresh_counters, dasc_debug_set_refresh_poll_limit,
+    dasc_conv_store, dasc_conv_load, dasc_plan_save, dasc_plan_load, dasc_refresh_counters, dasc_debug_set_refresh_poll_limit,
 )

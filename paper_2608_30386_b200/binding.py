@@ -28,7 +28,8 @@ OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_WORKSP
 # Every symbol include/dasc.h declares.
 EXPORTS = (
     "dasc_plan", "dasc_plan_destroy", "dasc_plan_info", "dasc_plan_horizon", "dasc_plan_mask",
-    "dasc_plan_window", "dasc_plan_layer_counts", "dasc_plan_layer_offsets", "dasc_pack", "dasc_restore",
+    "dasc_plan_window", "dasc_plan_layer_counts", "dasc_plan_layer_offsets", "dasc_plan_save_bytes", "dasc_plan_save",
+    "dasc_plan_load", "dasc_pack", "dasc_restore",
     "dasc_int8_slot_bytes", "dasc_pack_int8", "dasc_restore_int8",
     "dasc_padded_pool_floats", "dasc_pack_padded", "dasc_restore_padded", "dasc_checkpoint_bytes", "dasc_slot_budget",
     "dasc_tp_balance", "dasc_pack_tp", "dasc_restore_tp", "dasc_tp_head_permutation", "dasc_conv_store", "dasc_conv_load",
@@ -89,6 +90,9 @@ def lib() -> C.CDLL:
         for name in ("dasc_plan_horizon", "dasc_plan_mask", "dasc_plan_window", "dasc_plan_layer_counts",
                      "dasc_plan_layer_offsets"):
             getattr(L, name).argtypes = [C.c_void_p, C.c_void_p]
+        L.dasc_plan_save_bytes.argtypes = [C.c_void_p, C.POINTER(C.c_size_t)]
+        L.dasc_plan_save.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
+        L.dasc_plan_load.argtypes = [C.c_void_p, C.c_size_t, C.c_int32, C.POINTER(C.c_void_p)]
         L.dasc_pack.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64,
                                 C.c_void_p, C.c_int32, C.c_void_p]
         L.dasc_restore.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
@@ -227,6 +231,24 @@ def dasc_plan(kind, n_layers, n_v_heads, n_k_heads, d_k, d_v, A_log, dt_bias, *,
                     conv_bytes_per_ckpt)
     handle = C.c_void_p()
     _check(lib().dasc_plan(C.byref(desc), int(device), C.byref(handle)), "dasc_plan")
+    info = PlanInfo()
+    _check(lib().dasc_plan_info(handle, C.byref(info)), "dasc_plan_info")
+    return Plan(handle.value, info)
+
+
+def dasc_plan_save(plan: Plan) -> bytes:
+    """The plan as a self-contained blob (build it once where the weights are, load it in the serving processes)."""
+    n = C.c_size_t()
+    _check(lib().dasc_plan_save_bytes(plan.handle, C.byref(n)), "dasc_plan_save_bytes")
+    buf = C.create_string_buffer(n.value)
+    _check(lib().dasc_plan_save(plan.handle, buf, n.value), "dasc_plan_save")
+    return buf.raw
+
+
+def dasc_plan_load(blob: bytes, device: int = 0) -> Plan:
+    """Rebuild a plan from ``dasc_plan_save``'s blob; ``device=-1`` gives a host-only plan."""
+    handle = C.c_void_p()
+    _check(lib().dasc_plan_load(blob, len(blob), int(device), C.byref(handle)), "dasc_plan_load")
     info = PlanInfo()
     _check(lib().dasc_plan_info(handle, C.byref(info)), "dasc_plan_info")
     return Plan(handle.value, info)

@@ -4,6 +4,8 @@
 #include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
+#include <climits>
+#include <cstdint>
 #include <cstring>
 #include <new>
 
@@ -59,6 +61,29 @@ void free_device_tables(dasc_plan_s *p) {
 
 // The plan's index tables live on plan->info.device; a launch from another current device would hand the kernel
 // pointers of a GPU it may not be able to reach.
+// Upload the index tables of a host plan to `device` (the only device allocation this library makes).
+dasc_status_t attach_device(dasc_plan_s *p, int device) {
+  DeviceGuard guard(device);
+  if (!guard.ok) return DASC_ERR_CUDA;
+  p->info.device = device;
+  std::vector<uint8_t> keep(p->row_pos.size());
+  for (size_t i = 0; i < keep.size(); ++i) keep[i] = p->row_pos[i] >= 0 ? 1 : 0;
+  cudaError_t e = upload(&p->d_row_src, p->row_src.data(), p->row_src.size());
+  if (e == cudaSuccess) e = upload(&p->d_row_pos, p->row_pos.data(), p->row_pos.size());
+  if (e == cudaSuccess) e = upload(&p->d_row_keep, keep.data(), keep.size());
+  // packed row at which each layer starts: o_l in rows (a GDN unit is d_k rows)
+  const int64_t rows_per_unit = p->info.unit_floats / p->info.d_v;
+  std::vector<int32_t> row_off(p->layer_offset.size());
+  for (size_t l = 0; l < row_off.size(); ++l) row_off[l] = static_cast<int32_t>(p->layer_offset[l] * rows_per_unit);
+  if (e == cudaSuccess) e = upload(&p->d_layer_row_off, row_off.data(), row_off.size());
+  if (e != cudaSuccess) {
+    free_device_tables(p);
+    p->info.device = -1;
+    return e == cudaErrorMemoryAllocation ? DASC_ERR_ALLOC : DASC_ERR_CUDA;
+  }
+  return DASC_OK;
+}
+
 dasc_status_t check_device(const dasc_plan_t *plan) {
   if (!plan || plan->info.device < 0) return DASC_ERR_INVALID_ARG;
   int dev = -1;
@@ -125,26 +150,113 @@ dasc_status_t dasc_plan(const dasc_plan_desc_t *desc, int32_t device, dasc_plan_
     return st;
   }
   if (device >= 0) {
-    DeviceGuard guard(device);
-    if (!guard.ok) {
+    st = attach_device(p, device);
+    if (st != DASC_OK) {
       delete p;
-      return DASC_ERR_CUDA;
+      return st;
     }
-    p->info.device = device;
-    std::vector<uint8_t> keep(p->row_pos.size());
-    for (size_t i = 0; i < keep.size(); ++i) keep[i] = p->row_pos[i] >= 0 ? 1 : 0;
-    cudaError_t e = upload(&p->d_row_src, p->row_src.data(), p->row_src.size());
-    if (e == cudaSuccess) e = upload(&p->d_row_pos, p->row_pos.data(), p->row_pos.size());
-    if (e == cudaSuccess) e = upload(&p->d_row_keep, keep.data(), keep.size());
-    // packed row at which each layer starts: o_l in rows (a GDN unit is d_k rows)
-    const int64_t rows_per_unit = p->info.unit_floats / p->info.d_v;
-    std::vector<int32_t> row_off(p->layer_offset.size());
-    for (size_t l = 0; l < row_off.size(); ++l) row_off[l] = static_cast<int32_t>(p->layer_offset[l] * rows_per_unit);
-    if (e == cudaSuccess) e = upload(&p->d_layer_row_off, row_off.data(), row_off.size());
-    if (e != cudaSuccess) {
-      free_device_tables(p);
+  }
+  *out = p;
+  return DASC_OK;
+}
+
+// Saved plan: a flat little-endian blob { magic, version, sizeof(info), info, horizon[n], window[n], mask[n] };
+// everything else (layer counts, offsets, row tables) is re-derived from the mask when the blob is loaded.
+static constexpr uint64_t kPlanMagic = 0x314E4C5043534144ull;  // "DASCPLN1"
+struct PlanBlobHeader {
+  uint64_t magic;
+  uint32_t version, info_bytes;
+  int64_t n_units;
+};
+
+dasc_status_t dasc_plan_save_bytes(const dasc_plan_t *plan, size_t *out) {
+  if (!plan || !out) return DASC_ERR_INVALID_ARG;
+  const size_t n = plan->mask.size();
+  *out = sizeof(PlanBlobHeader) + sizeof(dasc_plan_info_t) + n * (sizeof(double) + sizeof(int64_t) + 1);
+  return DASC_OK;
+}
+
+dasc_status_t dasc_plan_save(const dasc_plan_t *plan, void *buf, size_t buf_bytes) {
+  size_t need = 0;
+  if (dasc_plan_save_bytes(plan, &need) != DASC_OK || !buf || buf_bytes < need) return DASC_ERR_INVALID_ARG;
+  const size_t n = plan->mask.size();
+  unsigned char *w = static_cast<unsigned char *>(buf);
+  const PlanBlobHeader h{kPlanMagic, 1u, static_cast<uint32_t>(sizeof(dasc_plan_info_t)), static_cast<int64_t>(n)};
+  dasc_plan_info_t info = plan->info;
+  info.device = -1;  // a saved plan belongs to no device
+  std::memcpy(w, &h, sizeof h); w += sizeof h;
+  std::memcpy(w, &info, sizeof info); w += sizeof info;
+  std::memcpy(w, plan->horizon.data(), n * sizeof(double)); w += n * sizeof(double);
+  std::memcpy(w, plan->window.data(), n * sizeof(int64_t)); w += n * sizeof(int64_t);
+  std::memcpy(w, plan->mask.data(), n);
+  return DASC_OK;
+}
+
+dasc_status_t dasc_plan_load(const void *buf, size_t bytes, int32_t device, dasc_plan_t **out) {
+  if (!out) return DASC_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!buf || bytes < sizeof(PlanBlobHeader) + sizeof(dasc_plan_info_t)) return DASC_ERR_INVALID_ARG;
+  const unsigned char *r = static_cast<const unsigned char *>(buf);
+  PlanBlobHeader h;
+  std::memcpy(&h, r, sizeof h); r += sizeof h;
+  if (h.magic != kPlanMagic || h.version != 1u || h.info_bytes != sizeof(dasc_plan_info_t) || h.n_units < 0)
+    return DASC_ERR_INVALID_ARG;
+  dasc_plan_info_t info;
+  std::memcpy(&info, r, sizeof info); r += sizeof info;
+  // the shape fields must be sane and agree with one another and with the blob's length before anything is sized by them
+  if (info.n_layers <= 0 || info.n_v_heads <= 0 || info.n_k_heads <= 0 || info.d_k <= 0 || info.d_v <= 0 || info.d_v % 4 ||
+      (info.kind != DASC_KDA && info.kind != DASC_GDN) || info.n_v_heads % info.n_k_heads)
+    return DASC_ERR_INVALID_ARG;
+  const int64_t n_l = static_cast<int64_t>(info.n_v_heads) * (info.kind == DASC_KDA ? info.d_k : 1);
+  const int64_t unit_floats = info.kind == DASC_KDA ? info.d_v : static_cast<int64_t>(info.d_k) * info.d_v;
+  const int64_t n = n_l * info.n_layers;
+  if (info.units_per_layer != n_l || info.unit_floats != unit_floats || info.units_total != n || h.n_units != n ||
+      static_cast<int64_t>(info.n_v_heads) * info.d_k * info.n_layers >= INT32_MAX)
+    return DASC_ERR_INVALID_ARG;
+  const size_t need = sizeof(PlanBlobHeader) + sizeof(dasc_plan_info_t) + static_cast<size_t>(n) * (sizeof(double) + sizeof(int64_t) + 1);
+  if (bytes < need) return DASC_ERR_INVALID_ARG;
+  dasc_plan_s *p = new (std::nothrow) dasc_plan_s();
+  if (!p) return DASC_ERR_ALLOC;
+  try {
+    p->info = info;
+    p->info.device = -1;
+    p->horizon.resize(n);
+    p->window.resize(n);
+    p->mask.resize(n);
+    std::memcpy(p->horizon.data(), r, n * sizeof(double)); r += n * sizeof(double);
+    std::memcpy(p->window.data(), r, n * sizeof(int64_t)); r += n * sizeof(int64_t);
+    std::memcpy(p->mask.data(), r, n);
+    p->layer_count.assign(info.n_layers, 0);
+    p->layer_offset.assign(info.n_layers + 1, 0);
+    int64_t r_max = 0;
+    for (int64_t l = 0; l < info.n_layers; ++l) {
+      int64_t c = 0;
+      for (int64_t u = 0; u < n_l; ++u) {
+        if (p->mask[l * n_l + u] > 1) throw 1;
+        c += p->mask[l * n_l + u];
+      }
+      p->layer_count[l] = c;
+      p->layer_offset[l + 1] = p->layer_offset[l] + c;
+      r_max = std::max(r_max, c);
+    }
+    // the counts the blob claims must be those of its mask
+    if (p->layer_offset[info.n_layers] != info.units_retained || r_max != info.r_max ||
+        info.slot_floats != info.units_retained * unit_floats ||
+        info.dense_floats_per_layer != static_cast<int64_t>(info.n_v_heads) * info.d_k * info.d_v)
+      throw 1;
+    dasc_plan_row_tables(p);
+  } catch (const std::bad_alloc &) {
+    delete p;
+    return DASC_ERR_ALLOC;
+  } catch (...) {
+    delete p;
+    return DASC_ERR_INVALID_ARG;
+  }
+  if (device >= 0) {
+    const dasc_status_t st = attach_device(p, device);
+    if (st != DASC_OK) {
       delete p;
-      return e == cudaErrorMemoryAllocation ? DASC_ERR_ALLOC : DASC_ERR_CUDA;
+      return st;
     }
   }
   *out = p;

@@ -34,6 +34,7 @@ struct dasc_plan_s {
 
 // plan_host.cpp
 dasc_status_t dasc_build_plan_host(const dasc_plan_desc_t *desc, dasc_plan_s *plan);
+void dasc_plan_row_tables(dasc_plan_s *plan);  // row_src / row_pos / packed_rows from info + mask
 
 // Section 4.3, second stage: where this rank's packed units live in the TP group's shared storage pool.
 constexpr int DASC_TP_MAX_RANKS = 16;

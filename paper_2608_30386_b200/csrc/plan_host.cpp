@@ -145,23 +145,6 @@ dasc_status_t dasc_build_plan_host(const dasc_plan_desc_t *d, dasc_plan_s *p) {
     if (!p->mask[u]) w_replay = std::max(w_replay, w);
   }
 
-  // --- row tables for the copy kernels --------------------------------------
-  p->rows_per_layer = rows_per_layer;
-  p->packed_rows = sum_r * rows_per_unit;
-  p->row_src.clear();
-  p->row_src.reserve(p->packed_rows);
-  p->row_pos.assign(L * rows_per_layer, -1);
-  for (int64_t l = 0; l < L; ++l) {
-    for (int64_t u = 0; u < n_l; ++u) {
-      if (!p->mask[l * n_l + u]) continue;
-      for (int64_t j = 0; j < rows_per_unit; ++j) {
-        const int64_t row = u * rows_per_unit + j;
-        p->row_pos[l * rows_per_layer + row] = static_cast<int32_t>(p->row_src.size());
-        p->row_src.push_back({static_cast<int32_t>(l), static_cast<int32_t>(row)});
-      }
-    }
-  }
-
   dasc_plan_info_t &o = p->info;
   o.kind = d->kind;
   o.n_layers = d->n_layers;
@@ -186,5 +169,30 @@ dasc_status_t dasc_build_plan_host(const dasc_plan_desc_t *d, dasc_plan_s *p) {
   o.w_max_used = cap;
   o.w_replay = static_cast<int64_t>(std::min(w_replay, w_clip));
   o.device = -1;
+  dasc_plan_row_tables(p);
   return DASC_OK;
+}
+
+// Row tables of the copy kernels from info + mask (also used when a saved plan is loaded): a row is d_v floats, a GDN
+// unit is d_k consecutive rows; row_src lists the retained rows in packed order, row_pos is its inverse (-1 = omitted).
+void dasc_plan_row_tables(dasc_plan_s *p) {
+  const dasc_plan_info_t &o = p->info;
+  const int64_t L = o.n_layers, n_l = o.units_per_layer;
+  const int64_t rows_per_unit = o.unit_floats / o.d_v;
+  const int64_t rows_per_layer = n_l * rows_per_unit;
+  p->rows_per_layer = rows_per_layer;
+  p->packed_rows = o.units_retained * rows_per_unit;
+  p->row_src.clear();
+  p->row_src.reserve(p->packed_rows);
+  p->row_pos.assign(L * rows_per_layer, -1);
+  for (int64_t l = 0; l < L; ++l) {
+    for (int64_t u = 0; u < n_l; ++u) {
+      if (!p->mask[l * n_l + u]) continue;
+      for (int64_t j = 0; j < rows_per_unit; ++j) {
+        const int64_t row = u * rows_per_unit + j;
+        p->row_pos[l * rows_per_layer + row] = static_cast<int32_t>(p->row_src.size());
+        p->row_src.push_back({static_cast<int32_t>(l), static_cast<int32_t>(row)});
+      }
+    }
+  }
 }

@@ -189,3 +189,30 @@ def test_mixed_per_head_ratios_explicit_mask():
     oracle.restore(oplan.mask, d, o_pool, slot, slots.numpy(), o_out, dense, L * dense, ids.numpy())
     np.testing.assert_array_equal(bits(d_pool), o_pool.view(np.uint32))
     np.testing.assert_array_equal(bits(d_out), o_out.view(np.uint32))
+
+
+@pytest.mark.gpu
+def test_a_saved_and_reloaded_plan_packs_and_restores_the_same_bits():
+    import torch
+    import paper_2608_30386_b200 as dasc
+    from paper_2608_30386_b200 import synth
+    from helpers import bits, make_plans
+    gen = synth.generator(91)
+    L, H, d = 3, 4, 32
+    rates = synth.decay_rates(gen, L, H, d, 1e-3, 1.0)
+    plan, oplan = make_plans(dasc.KDA, L, H, H, d, d, rates, sel=dasc.SEL_TOP_RATIO, scope=dasc.SCOPE_LAYER, keep_ratio=0.38)
+    again = dasc.dasc_plan_load(dasc.dasc_plan_save(plan), device=0)
+    assert again.device == 0 and again.units_retained == plan.units_retained
+    dense = H * d * d
+    state = synth.states(gen, (2, L, dense)).cuda()
+    ids = torch.arange(2, dtype=torch.int32, device="cuda")
+    pools, outs = [], []
+    for p in (plan, again):
+        pool = torch.zeros((2, int(p.slot_floats)), device="cuda")
+        out = torch.full_like(state, float("nan"))
+        dasc.dasc_pack(p, state, dense, L * dense, ids, pool, ids)
+        dasc.dasc_restore(p, pool, ids, out, dense, L * dense, ids)
+        pools.append(bits(pool))
+        outs.append(bits(out))
+    np.testing.assert_array_equal(pools[0], pools[1])
+    np.testing.assert_array_equal(outs[0], outs[1])

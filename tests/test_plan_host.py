@@ -178,3 +178,32 @@ def test_head_bundle_placement_matches_oracle(kind, H, hpb, T):
     assert U.max() <= contiguous.max()
     with pytest.raises(dasc.DascError):
         dasc.dasc_tp_head_permutation(p, 3, hpb)             # bundles do not divide among 3 ranks
+
+
+def test_plan_save_and_load_round_trip_and_reject_damaged_blobs():
+    rng = np.random.default_rng(77)
+    for kind, H, Hk, d in ((dasc.KDA, 4, 4, 16), (dasc.GDN, 8, 4, 8)):
+        L = 3
+        uph = d if kind == dasc.KDA else 1
+        A_log = np.log(_rates(rng, (L, H, uph)))
+        p = dasc.dasc_plan(kind, L, H, Hk, d, d, A_log, np.zeros_like(A_log), sel=dasc.SEL_TOP_RATIO,
+                           scope=dasc.SCOPE_MODEL, keep_ratio=0.37, conv_bytes_per_ckpt=4096, device=-1)
+        blob = dasc.dasc_plan_save(p)
+        q = dasc.dasc_plan_load(blob, device=-1)
+        for f, _ in binding.PlanInfo._fields_:
+            assert getattr(q.info, f) == getattr(p.info, f), f
+        np.testing.assert_array_equal(q.mask(), p.mask())
+        np.testing.assert_array_equal(q.horizon(), p.horizon())
+        np.testing.assert_array_equal(q.window(), p.window())
+        np.testing.assert_array_equal(q.layer_counts(), p.layer_counts())
+        np.testing.assert_array_equal(q.layer_offsets(), p.layer_offsets())
+        assert dasc.dasc_plan_save(q) == blob
+        # damaged blobs are refused: truncated, wrong magic, a mask that no longer matches the counts, a bad shape field
+        bad = [blob[:-1], b"X" + blob[1:], blob[:-1] + bytes([blob[-1] ^ 1])]
+        shape = bytearray(blob)
+        shape[24 + 4] ^= 0x7F                                   # n_layers inside the info struct
+        bad.append(bytes(shape))
+        for b in bad:
+            with pytest.raises(dasc.DascError) as e:
+                dasc.dasc_plan_load(b, device=-1)
+            assert e.value.status == binding.ERR_INVALID_ARG
