@@ -1,5 +1,5 @@
 // Suffix refresh, chunked form, on the Blackwell tensor cores (tcgen05 + TMEM), warp-specialised:
-// 32-token chunks, two CTAs resident per SM, three roles per CTA.
+// 32-token chunks, two CTAs resident per SM, four roles per CTA.
 //
 // Eq. 1 (transposed orientation) over a chunk of C = 32 tokens starting from S_0, with
 // G_t the running sum of the log-decay inside the chunk and m the chunk midpoint:
@@ -11,17 +11,22 @@
 //   S_C  = Diag(exp(G_C - G_m)) (S' + Kh^T U)
 //
 // Roles.  The operand tiles Kt, Qt, Kh depend on the token inputs only, not on the state, so they
-// are built one chunk ahead by four PRODUCER warps that read q, k and the log-decay straight from
-// global memory (their latency is off the critical path).  Eight CHAIN warps carry the
-// state-dependent sequence: state rescale -> triangular inverse -> right-hand side -> deltas ->
-// outputs.  One warp issues all tensor-core work.  The groups meet only at mbarriers.
+// are built one chunk ahead by four PRODUCER warps; their inputs land in the tiles they become (the
+// KDA log-decay by TMA, k and q by cp.async), off the critical path.  One TRIANGULAR warp forms
+// T = (I + A)^-1, also state-independent.  Eight CHAIN warps carry the state-dependent sequence:
+// state rescale -> right-hand side -> deltas -> outputs.  One warp issues all tensor-core work.
+// The groups meet only at mbarriers.  GDN (one scalar log-decay per token) keeps the decay out of
+// the products: MMA1 and MMA2 run on the raw k, q and the per-token factors are applied where A, P,
+// k S' and the outputs leave tensor memory.
 //   MMA1  [Kt;Qt] Kh^T            -> A (lanes 0-31) and P (lanes 32-63)         smem x smem
 //   MMA2  S'^T [Kt;Qt]^T          -> R^T | (Qt S')^T                            tmem x smem
 //   MMA3  RHS^T T^T               -> U^T      (RHS as a tf32 high/low pair)     tmem x smem
 //   MMA4  (Qt S')^T += U^T P^T    -> O^T                                         tmem x smem
 //   MMA5  S'^T      += U^T Kh     -> state    (U as a tf32 high/low pair)       tmem x smem
 // Buffers: the Kt/Qt and Kh tiles of chunk n+1 may be written once MMA2 of chunk n has completed
-// (MMA1 and MMA2 are their only readers); Kh^T, read last (MMA5), is double-buffered by chunk parity.
+// (MMA1 and MMA2 are their only readers); MMA5 contracts over the tokens and reads Kh as an MN-major
+// operand from a second tile (tf32 MN-major operands have a swizzle of their own), which, read last,
+// is double-buffered by chunk parity.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -483,7 +488,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
   } else if (warp >= 8) {
     // =============================== producer warps ===============================
     // warp = block of 32 channels; per half of the chunk, lane = (4 adjacent channels, 4 consecutive tokens), a 4 x 4
-    // tile, so that Kh can also be stored transposed.  The midpoint is the end of the first half: first-half
+    // tile.  The midpoint is the end of the first half: first-half
     // exponents are (local sum - the half's total), second-half exponents the local sums themselves.
     const int pw = warp - 8, ptid = tid - NCH;
     const int cq = lane & 7, tg = lane >> 3;
@@ -524,7 +529,7 @@ __global__ void __launch_bounds__(NT, 2) refresh_chunked_kernel(DascRefreshArgs 
         asm volatile("cp.async.commit_group;" ::: "memory");
       }
       // (b) raw k, q -> Kt/Qt tile, free once MMA2 of the previous chunk has completed; by then the chain warps
-      //     have also left the chunk before that one, whose parity buffers (post, Kh^T) are reused
+      //     have also left the chunk before that one, whose parity buffers (post, the MN-major Kh tile) are reused
       if (ch > 0) wait_bar(&misc->bar_ro, par ^ 1, misc, err);
 #pragma unroll
       for (int jj = 0; jj < 8; ++jj) {
